@@ -132,9 +132,9 @@ def time_oracle(coords, seed, sample_voxels):
     t0 = time.perf_counter()
     km = oracle.build_kmap(sub, 3, 1, 1, True)
     t1 = time.perf_counter()
-    oracle.forward(x, w, km["oft"])
+    ref = oracle.forward(x, w, km["oft"])
     t2 = time.perf_counter()
-    return len(sub), t1 - t0, t2 - t1, oracle.num_threads()
+    return len(sub), t1 - t0, t2 - t1, oracle.num_threads(), dict(coords=sub, x=x, w=w, ref=ref, pairs=len(km["pair_in"]))
 
 
 def run_reference(args):
@@ -146,7 +146,7 @@ def run_reference(args):
     n = 0
     threads = 1
     for i in range(args.warmup + args.steps):
-        n, tk, tf, threads = time_oracle(coords, 0, REFERENCE_SAMPLE_VOXELS)
+        n, tk, tf, threads, _ = time_oracle(coords, 0, REFERENCE_SAMPLE_VOXELS)
         if i >= args.warmup:
             total += tk + tf
     ms = 1e3 * total / args.steps
@@ -371,7 +371,18 @@ def run_ours(args):
         achieved = alg_bytes / (fwd * 1e-3) / 1e9
         t_hbm_us = alg_bytes / (peaks["hbm_gbs"] * 1e9) * 1e6
         t_mma_us = flops / (peaks["bf16_tflops"] * 1e12) * 1e6
-        cpu_n, cpu_tk, cpu_tf, cpu_threads = time_oracle(coords_np, seed, REFERENCE_SAMPLE_VOXELS)
+        cpu_n, cpu_tk, cpu_tf, cpu_threads, sample = time_oracle(coords_np, seed, REFERENCE_SAMPLE_VOXELS)
+        # Parity of the timed call on the timed workload (outside the timed region): the same spconv_layer call on the
+        # oracle's inputs, every output row against the oracle's fp64 result.
+        pk, py = binding.spconv_layer(torch.from_numpy(sample["coords"]).cuda(), torch.from_numpy(sample["x"]).to(torch.bfloat16).cuda(),
+                                      w, 1, 1, 3, True)
+        torch.cuda.synchronize()
+        p_status = binding.spconv_last_device_status(pk)
+        p_err = float(np.abs(py.float().cpu().numpy().astype(np.float64) - sample["ref"]).max() / np.abs(sample["ref"]).max())
+        parity = {"max_rel_err": p_err, "rows": int(py.shape[0]), "tolerance": 2e-2, "pairs_match": int(pk.total_pairs) == sample["pairs"],
+                  "device_status": p_status, "ok": bool(p_err <= 2e-2 and int(pk.total_pairs) == sample["pairs"] and p_status == 0),
+                  "what": "spconv_layer on sweep 0, all rows, vs the fp64 oracle (max-abs error / max |ref|)"}
+        pk.close()
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
             "ms_per_step": total_ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -396,6 +407,7 @@ def run_ours(args):
                          "peak_source": peaks["source"], "algorithmic_bytes": alg_bytes, "ms": fwd},
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms_max, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},
+            "parity": parity,
             "gpu_launches": OUR_LAUNCHES_PER_STEP * args.steps,
             "clocks": clocks,
             "wall_s": wall,

@@ -207,7 +207,9 @@ int spconv_layer_host(const int32_t* coords_host, int64_t n, const void* feats_h
  * forbidden.  spconv_build_kmap sizes and allocates its hash table per call; this entry point instead
  * probes a hash table kept in a fixed array inside the library (about 3 MiB, held by every GPU that loads
  * the library until the process exits) and writes straight into the caller's buffer.  It calls no
- * cudaMalloc / cudaFree, no stream-ordered allocator and no allocating library routine.
+ * cudaMalloc / cudaFree, no stream-ordered allocator and no allocating library routine.  (The array is part
+ * of the library's device code: the driver reserves it when it loads that code on a GPU, which with lazy
+ * module loading can be as late as the first call that launches a kernel of the library there.)
  *
  *   coords      device int32 [n][4] rows (b,x,y,z), 16-byte aligned, distinct, read only.
  *   n           0 <= n <= SPCONV_NOALLOC_MAX_VOXELS; larger inputs return SPCONV_ERR_TOO_LARGE

@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2402_07710_b200 import binding, workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -38,6 +39,28 @@ def test_two_calls_in_a_row_match_the_regular_entry_point():
         coords, want = _reference_table(coords_np, kernel, dilation)
         got = _noalloc_table(coords, kernel, dilation)
         assert torch.equal(got, want)                                          # integer table: bit-exact
+        # and against the CPU oracle's offset table (submanifold rows keep the input numbering on both sides)
+        ref = oracle.build_kmap(coords_np, kernel, 1, dilation, True)["oft"]
+        assert np.array_equal(got.cpu().numpy().T, ref)
+
+
+def test_second_call_takes_no_device_memory():
+    """Neither the caching allocator of the tensor library nor the driver's free-memory figure moves across a
+    call made with caller-owned tensors (the first call on a device may load the library's module; later ones
+    may not take anything)."""
+    coords_np = wl.shuffle_rows(wl.random_blob(4000, 22, seed=3), seed=4)
+    coords = torch.from_numpy(coords_np).cuda()
+    out = torch.empty(27, len(coords_np), dtype=torch.int32, device="cuda")
+    binding.spconv_subm_offset_table_noalloc(coords, 3, 1, out)
+    torch.cuda.synchronize()
+    reserved, allocated = torch.cuda.memory_reserved(), torch.cuda.memory_allocated()
+    free_before, _ = torch.cuda.mem_get_info()
+    binding.spconv_subm_offset_table_noalloc(coords, 3, 1, out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert torch.cuda.memory_reserved() == reserved and torch.cuda.memory_allocated() == allocated
+    assert free_after == free_before
+    assert np.array_equal(out.cpu().numpy().T, oracle.build_kmap(coords_np, 3, 1, 1, True)["oft"])
 
 
 def test_limits_and_input_errors_are_reported():
