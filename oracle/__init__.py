@@ -40,6 +40,9 @@ def _load():
         lib.oracle_kmap_build.restype = ctypes.c_void_p
         lib.oracle_kmap_build.argtypes = [i32p, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                           ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
+        lib.oracle_inverse_kmap_build.restype = ctypes.c_void_p
+        lib.oracle_inverse_kmap_build.argtypes = [i32p, ctypes.c_int64, i32p, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                                  ctypes.c_int, ctypes.POINTER(ctypes.c_int)]
         for name in ("oracle_kmap_n_out", "oracle_kmap_kvol", "oracle_kmap_total_pairs"):
             getattr(lib, name).restype = ctypes.c_int64
             getattr(lib, name).argtypes = [ctypes.c_void_p]
@@ -82,6 +85,29 @@ def build_kmap(coords, kernel: int, stride: int = 1, dilation: int = 1, submanif
                               int(bool(submanifold)), ctypes.byref(err))
     if not h:
         raise OracleError(err.value)
+    return _export(lib, h, c.shape[0])
+
+
+def build_inverse_kmap(fine, coarse, kernel: int, stride: int, dilation: int = 1) -> dict:
+    """Kernel map of the inverse (transposed) convolution of Sec. III-E.
+
+    ``fine`` are the positions before the strided convolution (the inverse layer's outputs, numbered as
+    given), ``coarse`` the positions after it (rows of the inverse layer's input features).  Same dict as
+    ``build_kmap`` with ``n_in = len(coarse)``, ``n_out = len(fine)``; ``oft[j, k]`` is the coarse row related
+    to fine row ``j`` through offset ``k`` or -1.
+    """
+    lib = _load()
+    f = np.ascontiguousarray(fine, dtype=np.int32).reshape(-1, 4)
+    c = np.ascontiguousarray(coarse, dtype=np.int32).reshape(-1, 4)
+    err = ctypes.c_int(0)
+    h = lib.oracle_inverse_kmap_build(_ptr(f, ctypes.c_int32), f.shape[0], _ptr(c, ctypes.c_int32), c.shape[0],
+                                      stride, dilation, kernel, ctypes.byref(err))
+    if not h:
+        raise OracleError(err.value)
+    return _export(lib, h, c.shape[0])
+
+
+def _export(lib, h, n_in: int) -> dict:
     try:
         n_out = lib.oracle_kmap_n_out(h)
         kvol = lib.oracle_kmap_kvol(h)
@@ -96,7 +122,7 @@ def build_kmap(coords, kernel: int, stride: int = 1, dilation: int = 1, submanif
                                _ptr(pair_out, ctypes.c_int32))
     finally:
         lib.oracle_kmap_free(h)
-    return dict(n_in=c.shape[0], n_out=int(n_out), kvol=int(kvol), out_coords=out_coords, oft=oft,
+    return dict(n_in=int(n_in), n_out=int(n_out), kvol=int(kvol), out_coords=out_coords, oft=oft,
                 offset_start=offset_start, pair_in=pair_in, pair_out=pair_out)
 
 

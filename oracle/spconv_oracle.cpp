@@ -14,6 +14,10 @@
 //     input position                                                       [Eq. 1-5, Sec. III-D]
 //   * Result: out[o][co] = sum_k sum_c in[OFT[o][k]][c] * w(k, c, co),
 //     skipping -1 entries                                                  [Algorithm 2]
+//   * Inverse (transposed) convolution: location table on the coarse index set
+//     ("indices2"), and for every position of the fine set ("indices1") the related
+//     coarse rows with their kernel offsets; the result is again Algorithm 2 over
+//     that table                                                           [Sec. III-E]
 //
 // Readings taken where the paper is silent (each also listed in the design notes):
 //   * orientation is correlation: offset k of output cell q looks at input
@@ -24,7 +28,13 @@
 //   * duplicate input coordinates are an error, not last-writer-wins;
 //   * output cells of a strided convolution are all cells touched by at least
 //     one input, numbered in lexicographic (b, x, y, z) order; o >= 0 on every axis;
-//   * weights are w[k][c][co] (row-major [K^3][Cin][Cout]).
+//   * weights are w[k][c][co] (row-major [K^3][Cin][Cout]);
+//   * inverse convolution: a fine position p is related to coarse cell q through offset kvec
+//     iff p = q*s + d*kvec - pad, i.e. exactly when p feeds q through kvec in the strided
+//     convolution with the same parameters; with K == s there is one such pair per fine position
+//     (the "singular weight and feature pair" of Sec. III-E), otherwise the related pairs are summed;
+//     a fine position without any related coarse row present gets a zero row; the fine rows keep
+//     the numbering of the fine index set.
 //
 // Accumulation is in double; inputs arrive as doubles converted exactly from
 // their storage type by the caller.
@@ -140,6 +150,66 @@ void* oracle_kmap_build(const int32_t* coords, int64_t n, int stride, int dilati
           km->oft[size_t(o) * kvol + k] = it->second;
           km->pair_in[k].push_back(it->second);
           km->pair_out[k].push_back(int32_t(o));
+        }
+  }
+  return km;
+}
+
+// Kernel map of the inverse convolution [Sec. III-E].  Stage 1: location table over the coarse
+// index set (fine -> "indices1" [n_fine][4], coarse -> "indices2" [n_coarse][4] in the paper's
+// words).  Stage 2: every fine position, every kernel offset: which coarse row is related through
+// that offset.  The returned map has n_in = n_coarse (rows of the input features), n_out = n_fine
+// (output row j = fine row j); its OFT row j lists, per offset k, the coarse row or -1.
+// Errors as for oracle_kmap_build (duplicates are checked in both sets).
+void* oracle_inverse_kmap_build(const int32_t* fine, int64_t n_fine, const int32_t* coarse, int64_t n_coarse,
+                                int stride, int dilation, int kernel, int* err) {
+  *err = 0;
+  if (n_fine < 0 || n_coarse < 0 || stride < 1 || dilation < 1 || kernel < 1) { *err = 1; return nullptr; }
+  const int K = kernel, s = stride, d = dilation;
+  const int64_t kvol = int64_t(K) * K * K;
+  const int pad = d * floor_half(K);
+
+  std::map<Coord, int32_t> lct2;   // location table of the coarse set
+  for (int64_t i = 0; i < n_coarse; ++i) {
+    Coord c{coarse[4 * i], coarse[4 * i + 1], coarse[4 * i + 2], coarse[4 * i + 3]};
+    for (int a = 0; a < 4; ++a) if (c[a] < 0) { *err = 2; return nullptr; }
+    if (!lct2.emplace(c, int32_t(i)).second) { *err = 3; return nullptr; }
+  }
+  {
+    std::map<Coord, int32_t> seen;
+    for (int64_t j = 0; j < n_fine; ++j) {
+      Coord c{fine[4 * j], fine[4 * j + 1], fine[4 * j + 2], fine[4 * j + 3]};
+      for (int a = 0; a < 4; ++a) if (c[a] < 0) { *err = 2; return nullptr; }
+      if (!seen.emplace(c, int32_t(j)).second) { *err = 3; return nullptr; }
+    }
+  }
+
+  auto* km = new Kmap;
+  km->kernel = K; km->stride = s; km->dilation = d; km->submanifold = 0;
+  km->n_in = n_coarse; km->n_out = n_fine; km->kvol = kvol;
+  km->pair_in.resize(kvol); km->pair_out.resize(kvol);
+  km->out_coords.resize(n_fine);
+  km->oft.assign(size_t(n_fine) * kvol, -1);
+  for (int64_t j = 0; j < n_fine; ++j) {
+    const int32_t* p = fine + 4 * j;
+    km->out_coords[j] = Coord{p[0], p[1], p[2], p[3]};
+    for (int kx = 0; kx < K; ++kx)
+      for (int ky = 0; ky < K; ++ky)
+        for (int kz = 0; kz < K; ++kz) {
+          const int64_t k = (int64_t(kx) * K + ky) * K + kz;       // Eq. 5
+          const int kv[3] = {kx, ky, kz};
+          Coord q{p[0], 0, 0, 0};
+          bool ok = true;
+          for (int a = 0; a < 3 && ok; ++a) {
+            const int num = p[a + 1] + pad - d * kv[a];              // q*s = p + pad - d*kvec
+            if (num < 0 || num % s != 0) ok = false; else q[a + 1] = num / s;
+          }
+          if (!ok) continue;
+          auto it = lct2.find(q);
+          if (it == lct2.end()) continue;
+          km->oft[size_t(j) * kvol + k] = it->second;
+          km->pair_in[k].push_back(it->second);
+          km->pair_out[k].push_back(int32_t(j));
         }
   }
   return km;

@@ -276,3 +276,119 @@ def test_workload_generators_are_seeded_and_sized():
     assert np.array_equal(torch.from_numpy(x).to(torch.bfloat16).float().numpy(), x)
     raw = np.random.default_rng(0).standard_normal(1000).astype(np.float32)
     assert np.array_equal(wl.round_to_dtype(raw, "bf16"), torch.from_numpy(raw).to(torch.bfloat16).float().numpy())
+
+
+# ----------------------------------------------------------------------------- inverse convolution (Sec. III-E)
+INVERSE_CASES = [(2, 2, 1), (3, 2, 1), (3, 1, 1), (3, 2, 2), (4, 2, 1), (3, 3, 1)]   # (K, s, d)
+
+
+def _fine_and_coarse(K, s, d, seed, n=240, extent=11):
+    fine = wl.shuffle_rows(wl.random_blob(n, extent, seed=seed, batches=2), seed=seed + 1)
+    coarse = oracle.build_kmap(fine, K, s, d, False)["out_coords"]     # the cells the strided convolution generates
+    coarse = wl.shuffle_rows(coarse, seed=seed + 2)                      # in an order of their own
+    return fine, coarse
+
+
+@pytest.mark.parametrize("K,s,d", INVERSE_CASES)
+def test_inverse_equals_dense_conv_transpose_at_every_fine_cell(K, s, d):
+    """The inverse convolution is the dense transposed convolution of the densified coarse features, read at the
+    fine positions: library conv_transpose3d in float64, weight[ci][co][kx][ky][kz] = W[k][ci][co]."""
+    rng = np.random.default_rng(100 + K * 7 + s * 3 + d)
+    fine, coarse = _fine_and_coarse(K, s, d, seed=K * 100 + s * 10 + d)
+    cin, cout = 3, 4
+    x = rng.standard_normal((len(coarse), cin))
+    w = rng.standard_normal((K ** 3, cin, cout))
+    km = oracle.build_inverse_kmap(fine, coarse, K, s, d)
+    assert km["n_in"] == len(coarse) and km["n_out"] == len(fine)
+    assert np.array_equal(km["out_coords"], fine)
+    y = oracle.forward(x, w, km["oft"])
+    pad = d * ((K - 1) // 2)
+    B = int(max(fine[:, 0].max(), coarse[:, 0].max())) + 1
+    grid = tuple(int(coarse[:, a].max()) + 1 for a in (1, 2, 3))
+    dense = torch.zeros(B, cin, *grid, dtype=torch.float64)
+    c = torch.from_numpy(coarse.astype(np.int64))
+    dense[c[:, 0], :, c[:, 1], c[:, 2], c[:, 3]] = torch.from_numpy(x)
+    wd = torch.from_numpy(w).reshape(K, K, K, cin, cout).permute(3, 4, 0, 1, 2).contiguous()
+    up = torch.nn.functional.conv_transpose3d(dense, wd, stride=s, padding=pad, dilation=d, output_padding=s - 1 if s > 1 else 0).numpy()
+    for j, (b, px, py, pz) in enumerate(fine.tolist()):
+        inside = px < up.shape[2] and py < up.shape[3] and pz < up.shape[4]
+        want = up[b, :, px, py, pz] if inside else np.zeros(cout)
+        assert np.allclose(y[j], want, rtol=0, atol=1e-12), (j, fine[j])
+
+
+@pytest.mark.parametrize("K,s,d", INVERSE_CASES)
+def test_inverse_is_the_adjoint_of_the_strided_convolution(K, s, d):
+    """<conv(x), y> = <x, inverse(y)> when the inverse layer uses the transposed weight slices: the defining
+    property of a transposed convolution, checked without looking at either kernel map."""
+    rng = np.random.default_rng(K * 31 + s * 5 + d)
+    fine, _ = _fine_and_coarse(K, s, d, seed=K * 50 + s * 9 + d)
+    fwd = oracle.build_kmap(fine, K, s, d, False)
+    coarse = fwd["out_coords"]
+    cf, cc = 3, 2
+    w = rng.standard_normal((K ** 3, cf, cc))
+    x = rng.standard_normal((len(fine), cf))
+    y = rng.standard_normal((len(coarse), cc))
+    conv_x = oracle.forward(x, w, fwd["oft"])                                  # [n_coarse, cc]
+    inv = oracle.build_inverse_kmap(fine, coarse, K, s, d)
+    inv_y = oracle.forward(y, np.ascontiguousarray(w.transpose(0, 2, 1)), inv["oft"])   # [n_fine, cf]
+    assert abs((conv_x * y).sum() - (x * inv_y).sum()) <= 1e-10 * max(1.0, abs((conv_x * y).sum()))
+
+
+@pytest.mark.parametrize("K,s,d", INVERSE_CASES)
+def test_inverse_kmap_brute_force_and_role_swap(K, s, d):
+    """Brute force over all (fine, coarse, offset) triples with explicit coordinate comparison; and the same
+    relation as the strided convolution's with the roles of the two sets swapped."""
+    fine, coarse = _fine_and_coarse(K, s, d, seed=K * 13 + s + d, n=90, extent=8)
+    pad = d * ((K - 1) // 2)
+    inv = oracle.build_inverse_kmap(fine, coarse, K, s, d)
+    want = set()
+    for j, (fb, fx, fy, fz) in enumerate(fine.tolist()):
+        for q, (cb, cx, cy, cz) in enumerate(coarse.tolist()):
+            for k, (kx, ky, kz) in enumerate(itertools.product(range(K), repeat=3)):
+                if fb == cb and fx == cx * s + d * kx - pad and fy == cy * s + d * ky - pad and fz == cz * s + d * kz - pad:
+                    want.add((q, j, k))
+    got = triples_of(_canon(inv, relabel=False))
+    assert got == want
+    from_table = {(int(inv["oft"][j, k]), j, k) for j in range(len(fine)) for k in range(K ** 3) if inv["oft"][j, k] >= 0}
+    assert from_table == want
+    # role swap: (i_fine, o_coarse, k) of the strided map <=> (o_coarse, i_fine, k) here
+    fwd = oracle.build_kmap(fine, K, s, d, False)
+    index_of = {tuple(c): i for i, c in enumerate(coarse.tolist())}
+    relabel = [index_of[tuple(c)] for c in fwd["out_coords"].tolist()]
+    swapped = {(relabel[o], i, k) for (i, o, k) in triples_of(_canon(fwd, relabel=False))}
+    assert swapped == want
+
+
+@pytest.mark.parametrize("s", [2, 1])
+def test_inverse_kernel_equals_stride_is_one_pair_per_fine_position(s):
+    """K == s with zero padding (K = 2 or 1 under pad = floor((K-1)/2)): Eq. 1-5 give every fine position exactly
+    one coarse parent floor(p/s) and the offset p mod s, so each output row is a single weight-feature product,
+    as Sec. III-E says."""
+    fine, coarse = _fine_and_coarse(s, s, 1, seed=77)
+    inv = oracle.build_inverse_kmap(fine, coarse, s, s, 1)
+    assert (np.sum(inv["oft"] >= 0, axis=1) == 1).all() and inv["offset_start"][-1] == len(fine)
+    index_of = {tuple(c): i for i, c in enumerate(coarse.tolist())}
+    p = fine[:, 1:].astype(np.int64)
+    off = p - (p // s) * s
+    k = off[:, 0] * s * s + off[:, 1] * s + off[:, 2]
+    for j in range(len(fine)):
+        parent = index_of[(int(fine[j, 0]), *(p[j] // s).tolist())]
+        assert inv["oft"][j, k[j]] == parent
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((len(coarse), 2)); w = rng.standard_normal((s ** 3, 2, 3))
+    y = oracle.forward(x, w, inv["oft"])
+    for j in range(len(fine)):
+        assert np.allclose(y[j], x[inv["oft"][j, k[j]]] @ w[k[j]], rtol=0, atol=1e-13)
+
+
+def test_inverse_missing_parent_gives_zero_row_and_errors():
+    fine = np.array([[0, 4, 4, 4], [0, 9, 9, 9]], np.int32)
+    coarse = np.array([[0, 2, 2, 2]], np.int32)                 # the parent of the first position only
+    inv = oracle.build_inverse_kmap(fine, coarse, 2, 2, 1)
+    assert inv["oft"][0].tolist().count(-1) == 7 and inv["oft"][0, 0] == 0 and (inv["oft"][1] == -1).all()
+    y = oracle.forward(np.ones((1, 2)), np.ones((8, 2, 2)), inv["oft"])
+    assert (y[1] == 0).all() and (y[0] == 2).all()
+    with pytest.raises(oracle.OracleError):
+        oracle.build_inverse_kmap(np.array([[0, 1, 1, 1], [0, 1, 1, 1]], np.int32), coarse, 2, 2, 1)
+    with pytest.raises(oracle.OracleError):
+        oracle.build_inverse_kmap(fine, np.array([[0, -1, 0, 0]], np.int32), 2, 2, 1)
