@@ -85,6 +85,8 @@ typedef struct {
   const int64_t* offset_start; /* HOST [kvol+1], owned by the handle */
   const int32_t* tile_rows;    /* device [n_tiles][128]: output row processed at each tile slot, -1 = padding */
   int64_t tile_blocks;         /* number of non-empty (tile, offset) blocks in the tensor-core plan */
+  int32_t inverse;             /* 1 for a map from spconv_build_inverse_kmap */
+  int32_t reserved;
 } spconv_kmap_info_t;
 
 /*
@@ -111,6 +113,31 @@ typedef struct {
  */
 int spconv_build_kmap(const int32_t* coords, int64_t n, int stride, int dilation, int kernel_size,
                       int submanifold, void* cuda_stream, spconv_kmap_t** kmap_out);
+
+/*
+ * Build the kernel map of an inverse (transposed) convolution, the up-sampling counterpart of a strided layer.
+ * [Sec. III-E: location table over the index set after the convolution ("indices2"), then for every position of
+ * the index set before it ("indices1") the related location in indices2 and its offset in the kernel]
+ *
+ *   fine_coords    device int32 [n_fine][4] rows (b,x,y,z): the positions BEFORE the strided convolution.  They are
+ *                  the output rows of the inverse layer, numbered as given.  16-byte aligned, distinct (not
+ *                  checked), read only.
+ *   coarse_coords  device int32 [n_coarse][4]: the positions AFTER it (for instance the out_coords of the strided
+ *                  layer's map, as a device pointer, no copy needed).  Row i is row i of the inverse layer's input
+ *                  features.  16-byte aligned, distinct (checked), read only.
+ *   stride, dilation, kernel_size   those of the strided convolution being inverted.
+ * Fine position p is related to coarse cell q through offset kvec iff p = q*stride + dilation*kvec - pad,
+ * pad = dilation*floor((K-1)/2): exactly the pairs of the strided convolution with the two roles swapped.  With
+ * kernel_size == stride every fine position has one related cell (o = floor(p/s), offset p mod s, Eq. 1-5) and its
+ * output row is the single product the paper describes; otherwise the related products are summed.  A fine
+ * position none of whose related cells is in coarse_coords gets an all-zero output row.
+ * The handle has n_in = n_coarse, n_out = n_fine, out_coords = a copy of fine_coords, and is used with
+ * spconv_forward like any other: feats [n_coarse][cin], weights [K^3][cin][cout] (for the adjoint of a strided
+ * layer pass that layer's W_k transposed), out [n_fine][cout].
+ * Host wait, scratch memory, stream semantics and errors as for spconv_build_kmap.
+ */
+int spconv_build_inverse_kmap(const int32_t* fine_coords, int64_t n_fine, const int32_t* coarse_coords, int64_t n_coarse,
+                              int stride, int dilation, int kernel_size, void* cuda_stream, spconv_kmap_t** kmap_out);
 
 /* Describe a kernel map.  `info` is host memory; the pointers inside stay valid until destroy. */
 int spconv_kmap_info(const spconv_kmap_t* kmap, spconv_kmap_info_t* info);

@@ -21,7 +21,7 @@ _TORCH_DTYPE = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
 DTYPE_BY_NAME = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
 
 EXPORTS = (
-    "spconv_build_kmap", "spconv_kmap_info", "spconv_kmap_destroy", "spconv_forward", "spconv_forward_algo",
+    "spconv_build_kmap", "spconv_build_inverse_kmap", "spconv_kmap_info", "spconv_kmap_destroy", "spconv_forward", "spconv_forward_algo",
     "spconv_last_device_status", "spconv_layer", "spconv_layer_host", "spconv_strerror", "spconv_subm_offset_table_noalloc",
 )
 NOALLOC_MAX_VOXELS = 131072
@@ -41,6 +41,7 @@ class _KmapInfo(ctypes.Structure):
         ("out_coords", ctypes.c_void_p), ("nbr", ctypes.c_void_p), ("pair_in", ctypes.c_void_p),
         ("pair_out", ctypes.c_void_p), ("offset_start", ctypes.POINTER(ctypes.c_int64)),
         ("tile_rows", ctypes.c_void_p), ("tile_blocks", ctypes.c_int64),
+        ("inverse", ctypes.c_int32), ("reserved", ctypes.c_int32),
     ]
 
 
@@ -60,6 +61,8 @@ def load() -> ctypes.CDLL:
         vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
         lib.spconv_build_kmap.restype = i32
         lib.spconv_build_kmap.argtypes = [vp, i64, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        lib.spconv_build_inverse_kmap.restype = i32
+        lib.spconv_build_inverse_kmap.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, ctypes.POINTER(vp)]
         lib.spconv_kmap_info.restype = i32
         lib.spconv_kmap_info.argtypes = [vp, ctypes.POINTER(_KmapInfo)]
         lib.spconv_kmap_destroy.restype = None
@@ -120,7 +123,7 @@ class Kmap:
             raise SpconvError(st, "spconv_kmap_info")
         self._info = info
         for name in ("kernel_size", "stride", "dilation", "submanifold", "kvol", "n_tiles", "n_in", "n_out",
-                     "total_pairs", "tile_blocks"):
+                     "total_pairs", "tile_blocks", "inverse"):
             setattr(self, name, int(getattr(info, name)))
         self._offset_start = None   # converted on first use: the build sits on the latency path of a layer
 
@@ -182,6 +185,23 @@ def spconv_build_kmap(coords: torch.Tensor, stride: int = 1, dilation: int = 1, 
                                   ctypes.c_void_p(_stream_ptr(stream)), ctypes.byref(h))
     if st != 0:
         raise SpconvError(st, "spconv_build_kmap")
+    return Kmap(h.value)
+
+
+def spconv_build_inverse_kmap(fine_coords: torch.Tensor, coarse_coords: torch.Tensor, stride: int, dilation: int = 1,
+                              kernel_size: int = 3, stream=None) -> Kmap:
+    """Kernel map of the inverse (transposed) convolution: output rows are ``fine_coords`` (positions before the
+    strided layer), input rows ``coarse_coords`` (positions after it); both device ``int32 [n, 4]``."""
+    for c in (fine_coords, coarse_coords):
+        if not (c.is_cuda and c.dtype == torch.int32 and c.dim() == 2 and c.shape[1] == 4 and c.is_contiguous()):
+            raise ValueError("coordinates must be contiguous CUDA int32 tensors of shape [n, 4]")
+    h = ctypes.c_void_p(None)
+    st = load().spconv_build_inverse_kmap(ctypes.c_void_p(fine_coords.data_ptr() if fine_coords.numel() else 0), fine_coords.shape[0],
+                                          ctypes.c_void_p(coarse_coords.data_ptr() if coarse_coords.numel() else 0),
+                                          coarse_coords.shape[0], int(stride), int(dilation), int(kernel_size),
+                                          ctypes.c_void_p(_stream_ptr(stream)), ctypes.byref(h))
+    if st != 0:
+        raise SpconvError(st, "spconv_build_inverse_kmap")
     return Kmap(h.value)
 
 

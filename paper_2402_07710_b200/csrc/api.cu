@@ -50,6 +50,22 @@ int spconv_build_kmap(const int32_t* coords, int64_t n, int stride, int dilation
   return spconv_build_kmap_hooked(coords, n, stride, dilation, kernel_size, submanifold, cuda_stream, kmap_out, nullptr);
 }
 
+int spconv_build_inverse_kmap(const int32_t* fine_coords, int64_t n_fine, const int32_t* coarse_coords, int64_t n_coarse,
+                              int stride, int dilation, int kernel_size, void* cuda_stream, spconv_kmap_t** kmap_out) {
+  if (kmap_out == nullptr) return SPCONV_ERR_INVALID_ARG;
+  *kmap_out = nullptr;
+  if (n_fine < 0 || n_coarse < 0 || stride < 1 || dilation < 1 || kernel_size < 1) return SPCONV_ERR_INVALID_ARG;
+  if (kernel_size > 16 || stride > 4096 || dilation > 4096) return SPCONV_ERR_INVALID_ARG;
+  if ((n_fine > 0 && fine_coords == nullptr) || (n_coarse > 0 && coarse_coords == nullptr)) return SPCONV_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(fine_coords) & 15u) || (reinterpret_cast<uintptr_t>(coarse_coords) & 15u)) return SPCONV_ERR_INVALID_ARG;
+  const int64_t kvol = int64_t(kernel_size) * kernel_size * kernel_size;
+  if (n_fine * kvol > int64_t(2000000000) || n_coarse > int64_t(2000000000)) return SPCONV_ERR_TOO_LARGE;
+  // a never-null query pointer selects the inverse path even when there are no fine rows
+  static const int32_t none[4] = {0, 0, 0, 0};
+  return build_kmap_impl(coarse_coords, n_coarse, stride, dilation, kernel_size, 0, static_cast<cudaStream_t>(cuda_stream), kmap_out,
+                         nullptr, fine_coords != nullptr ? fine_coords : none, n_fine);
+}
+
 int spconv_kmap_info(const spconv_kmap_t* km, spconv_kmap_info_t* info) {
   if (km == nullptr || info == nullptr) return SPCONV_ERR_INVALID_ARG;
   std::memset(info, 0, sizeof(*info));
@@ -60,6 +76,7 @@ int spconv_kmap_info(const spconv_kmap_t* km, spconv_kmap_info_t* info) {
   info->pair_in = km->d.pair_in; info->pair_out = km->d.pair_out;
   info->offset_start = km->offset_start.data();
   info->tile_rows = km->d.tile_rows; info->tile_blocks = km->tile_blocks;
+  info->inverse = km->inverse;
   return SPCONV_OK;
 }
 

@@ -41,7 +41,7 @@ struct KmapDeviceArrays {
 }  // namespace spconv
 
 struct spconv_kmap {
-  int kernel = 0, stride = 0, dilation = 0, submanifold = 0, kvol = 0;
+  int kernel = 0, stride = 0, dilation = 0, submanifold = 0, inverse = 0, kvol = 0;
   int device = 0;
   cudaStream_t stream = nullptr;      // stream the map was built on; its memory is released in this stream's order
   int mask_words = 1;
@@ -57,8 +57,11 @@ namespace spconv {
 // before_wait (optional, submanifold maps only): called once every kernel of the build has been enqueued and before
 // the host waits for the device's report, with the handle's sizes and device pointers set (pair count and block
 // count are not known yet); what it enqueues on the stream runs behind the build without a host round trip between.
+// fine_coords (optional): builds the map of the inverse convolution instead: `coords` are then the coarse positions
+// (rows of the input features), fine_coords [n_fine][4] the output rows, and submanifold must be 0.
 int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, int kernel, int submanifold,
-                    cudaStream_t stream, spconv_kmap** out, const std::function<int(spconv_kmap*)>* before_wait = nullptr);
+                    cudaStream_t stream, spconv_kmap** out, const std::function<int(spconv_kmap*)>* before_wait = nullptr,
+                    const int32_t* fine_coords = nullptr, int64_t n_fine = 0);
 void destroy_kmap_impl(spconv_kmap* km);
 
 // forward_simt.cu

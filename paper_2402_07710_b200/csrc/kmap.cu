@@ -32,6 +32,19 @@ __device__ __forceinline__ void chain_begin() {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
+#ifdef SPCONV_KMAP_TIMELINE
+// Development builds: globaltimer stamps of block 0 / thread 0 at the start (after the dependency wait) and the end of
+// the build's kernels, slot 2 * id and 2 * id + 1.
+__device__ unsigned long long g_kmap_timeline[32];
+__device__ __forceinline__ void tl_stamp(int slot) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); g_kmap_timeline[slot] = t; }
+}
+#define SPCONV_TL(slot) tl_stamp(slot)
+#define SPCONV_TL_RAW(slot, t) g_kmap_timeline[slot] = (t)
+#else
+#define SPCONV_TL(slot)
+#define SPCONV_TL_RAW(slot, t)
+#endif
 template <class... Params, class... Args>
 cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
   cudaLaunchConfig_t config = {};
@@ -46,7 +59,6 @@ cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, cud
   config.numAttrs = 1;
   return cudaLaunchKernelEx(&config, kernel, Params(args)...);
 }
-
 
 constexpr int kBlock = 256;
 
@@ -81,19 +93,22 @@ OffsetIndex make_offset_index(int K) {
   return t;
 }
 
+// 32-bit mix of the two key halves (two independent multiplies, then one round of xor-shift-multiply): a short
+// dependency chain, where a 64-bit finaliser's two dependent wide multiplies were most of a lookup's instructions.
 __device__ __forceinline__ uint32_t hash_key(uint64_t k) {
-  k ^= k >> 33; k *= 0xff51afd7ed558ccdULL;
-  k ^= k >> 33; k *= 0xc4ceb9fe1a85ec53ULL;
-  k ^= k >> 33;
-  return uint32_t(k);
+  uint32_t h = (uint32_t(k) * 0x9E3779B1u) ^ (uint32_t(k >> 32) * 0x85EBCA77u);
+  h ^= h >> 15; h *= 0x2C1B3C6Du; h ^= h >> 12;
+  return h;
 }
 
 // Open addressing, linear probing.  Returns the slot that holds `key` (inserting it if absent) or -1
 // if the bounded probe sequence found neither the key nor a free slot.  *was_present tells which.
+// A slot is STRIDE 64-bit words wide and starts with its key.
+template <int STRIDE>
 __device__ __forceinline__ int table_insert(uint64_t* keys, uint32_t capmask, uint64_t key, bool* was_present) {
   uint32_t slot = hash_key(key) & capmask;
   for (uint32_t probe = 0; probe <= capmask; ++probe) {
-    unsigned long long old = atomicCAS(reinterpret_cast<unsigned long long*>(keys + slot),
+    unsigned long long old = atomicCAS(reinterpret_cast<unsigned long long*>(keys + size_t(slot) * STRIDE),
                                        (unsigned long long)kEmptyKey, (unsigned long long)key);
     if (old == kEmptyKey) { *was_present = false; return int(slot); }
     if (old == key) { *was_present = true; return int(slot); }
@@ -102,39 +117,61 @@ __device__ __forceinline__ int table_insert(uint64_t* keys, uint32_t capmask, ui
   return -1;
 }
 
-__device__ __forceinline__ int table_find(const uint64_t* __restrict__ keys, const int32_t* __restrict__ vals,
-                                          uint32_t capmask, uint64_t key) {
+// The location table keeps key and row index side by side in 16-byte slots (key | row | unused), so that a lookup
+// that hits costs one memory request: the row arrives with the key it is compared against.
+struct __align__(16) LocSlot { uint64_t key; int32_t row; int32_t unused; };
+__device__ __forceinline__ LocSlot load_slot(const LocSlot* __restrict__ table, uint32_t slot) {
+  const ulonglong2 raw = __ldg(reinterpret_cast<const ulonglong2*>(table) + slot);
+  LocSlot s;
+  s.key = raw.x; s.row = int32_t(uint32_t(raw.y)); s.unused = 0;
+  return s;
+}
+__device__ __forceinline__ int table_find(const LocSlot* __restrict__ table, uint32_t capmask, uint64_t key) {
   uint32_t slot = hash_key(key) & capmask;
   for (uint32_t probe = 0; probe <= capmask; ++probe) {
-    const uint64_t k = __ldg(keys + slot);
-    if (k == key) return __ldg(vals + slot);
-    if (k == kEmptyKey) return -1;
+    const LocSlot s = load_slot(table, slot);
+    if (s.key == key) return s.row;
+    if (s.key == kEmptyKey) return -1;
     slot = (slot + 1) & capmask;
   }
   return -1;
 }
 
+// Occupancy filter in front of the location table: one bit per cell of a 256 x 256 x 64 window onto which all
+// positions are folded (x also shifted by the batch index), CLEAR where some inserted position folds to the cell
+// (so that the byte pattern that empties the table's keys, 0xFF, also empties the filter).  A set bit proves that
+// the table does not hold the position: five of six neighbour lookups of a surface-like input end there, with one
+// read that neighbouring threads share (z runs along the bits of a word, y along the words of a line), instead of
+// a read of a hashed, unshared table slot.  A clear bit proves nothing; the table decides.
+constexpr uint32_t kOccWords = 131072;   // 4 Mi bits
+__device__ __forceinline__ uint32_t occ_word(int b, int x, int y, int z) {
+  return ((uint32_t(x + 37 * b) & 255u) << 9) | ((uint32_t(y) & 255u) << 1) | ((uint32_t(z) >> 5) & 1u);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Location table: coordinate -> input row.  One int4 load per voxel.
-__global__ void k_insert(const int4* __restrict__ coords, int n, uint64_t* keys, int32_t* vals, uint32_t capmask,
-                         uint32_t* status, int4* __restrict__ coords_copy) {
+__global__ void k_insert(const int4* __restrict__ coords, int n, LocSlot* table, uint32_t capmask,
+                         uint32_t* status, int4* __restrict__ coords_copy, uint32_t* __restrict__ occ = nullptr) {
   chain_begin();
+  SPCONV_TL(0);
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const int4 c = coords[i];
   if (coords_copy != nullptr) coords_copy[i] = c;   // submanifold: the output coordinates are the input's
   if (!(in_range(c.x) && in_range(c.y) && in_range(c.z) && in_range(c.w))) { atomicOr(status, kDevCoordRange); return; }
   bool present;
-  const int slot = table_insert(keys, capmask, pack_key(c.x, c.y, c.z, c.w), &present);
+  const int slot = table_insert<2>(reinterpret_cast<uint64_t*>(table), capmask, pack_key(c.x, c.y, c.z, c.w), &present);
   if (slot < 0) { atomicOr(status, kDevTableFull); return; }
   if (present) { atomicOr(status, kDevDuplicate); return; }
-  vals[slot] = i;
+  table[slot].row = i;
+  if (occ != nullptr) atomicAnd(occ + occ_word(c.x, c.y, c.z, c.w), ~(1u << (c.w & 31)));
+  SPCONV_TL(1);
 }
 
 // Offset table for submanifold convolution, offset-major: nbr[k][j] = input row at c_j + d*(kvec - r), or -1.
 // grid = (ceil(n/256), kvol).  Also counts the hits of each block for the pair compaction.
-__global__ void k_subm_probe(const int4* __restrict__ coords, int n, int K, int dil, const uint64_t* __restrict__ keys,
-                             const int32_t* __restrict__ vals, uint32_t capmask, int32_t* __restrict__ nbr,
+__global__ void k_subm_probe(const int4* __restrict__ coords, int n, int K, int dil, const LocSlot* __restrict__ table,
+                             uint32_t capmask, int32_t* __restrict__ nbr,
                              int32_t* __restrict__ blockcnt, unsigned* __restrict__ offset_cnt, const __grid_constant__ OffsetIndex index) {
   chain_begin();
   const int k = blockIdx.y;
@@ -148,7 +185,7 @@ __global__ void k_subm_probe(const int4* __restrict__ coords, int n, int K, int 
     const int4 c = coords[j];
     const int x = c.y + dx, y = c.z + dy, z = c.w + dz;
     if ((dx | dy | dz) == 0) v = j;
-    else if (in_range(x) && in_range(y) && in_range(z)) v = table_find(keys, vals, capmask, pack_key(c.x, x, y, z));
+    else if (in_range(x) && in_range(y) && in_range(z)) v = table_find(table, capmask, pack_key(c.x, x, y, z));
     nbr[size_t(k) * n + j] = v;
   }
   const int cnt = __syncthreads_count(v >= 0);
@@ -158,60 +195,180 @@ __global__ void k_subm_probe(const int4* __restrict__ coords, int n, int K, int 
   }
 }
 
-// The same table, K offsets per thread: thread j of block (x, ab) takes the K offsets k = ab*K + c, c = 0..K-1 (a
-// line along z), and issues their first table reads together, so that it has K independent requests in flight
-// instead of one (the one-offset kernel spends its time waiting for dependent round trips to L2).
-// grid = (ceil(n/256), K*K).
-template <int KZ>
-__global__ void k_subm_probe_line(const int4* __restrict__ coords, int n, int dil, const uint64_t* __restrict__ keys,
-                                  const int32_t* __restrict__ vals, uint32_t capmask, int32_t* __restrict__ nbr,
-                                  int32_t* __restrict__ blockcnt, unsigned* __restrict__ offset_cnt, const __grid_constant__ OffsetIndex index) {
+// ---------------------------------------------------------------------------------------------
+// Offset table, every offset of one output row per thread (kernel volumes up to 32).
+//   MODE 0, submanifold (Sec. III-C.2): row j looks at p_j + d*(kvec - r); the centre offset is j itself.
+//   MODE 1, inverse convolution (Sec. III-E): the table was built over the coarse positions; fine position p_j is
+//           related to coarse cell (p_j + pad - d*kvec) / s through offset kvec where that is a whole cell >= 0.
+// The occupancy filter is consulted for every offset first (see occ_word); the table lookups of the offsets it
+// does not rule out follow four at a time.  The table is written in two layouts: offset-major nbr[k][j] (the caller's
+// view, the pair emission and the CUDA-core forward read it along j) and row-major rows of 32 entries
+// nbr_rows[j][k] (the paper's OFT layout; the tile plan reads whole rows of permuted j).  row_mask[j] has bit k
+// set where the row has an input through offset k.  Per block and offset the number of hits goes to blockcnt
+// (the pair emission's bases), per offset the total to offset_cnt.
+template <int K, int MODE>
+__global__ void __launch_bounds__(kBlock)
+k_probe_rows(const int4* __restrict__ qcoords, int nq, int dil, int stride, const LocSlot* __restrict__ table,
+             uint32_t capmask, const uint32_t* __restrict__ occ, int32_t* __restrict__ nbr,
+             int32_t* __restrict__ nbr_rows, uint32_t* __restrict__ row_mask, int32_t* __restrict__ blockcnt,
+             unsigned* __restrict__ offset_cnt, int4* __restrict__ coords_copy, uint32_t* __restrict__ status) {
   chain_begin();
-  constexpr int r = (KZ - 1) / 2;
-  const int ab = blockIdx.y, k0 = ab * KZ;
+  SPCONV_TL(2);
+  constexpr int KV = K * K * K;
+  static_assert(KV <= 32, "kernel volume");
+  constexpr int r = (K - 1) / 2;
+  __shared__ int s_v[KV][kBlock];   // the row's entries, written at run-time offsets, read back by the same thread
+  __shared__ unsigned s_cnt[32];
+  if (threadIdx.x < 32) s_cnt[threadIdx.x] = 0u;
+  __syncthreads();
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int j = blockIdx.x * kBlock + tid;
+  const bool live = j < nq;
+  int4 c = make_int4(0, 0, 0, 0);
+  if (live) {
+    c = qcoords[j];
+    if (coords_copy != nullptr) coords_copy[j] = c;
+  }
+  bool usable = live;
+  if (MODE == 1 && live && !(in_range(c.x) && in_range(c.y) && in_range(c.z) && in_range(c.w))) {
+    atomicOr(status, kDevCoordRange);
+    usable = false;
+  }
+  const int pad = dil * r;
+  const bool pow2 = (stride & (stride - 1)) == 0;
+  const int shift = __ffs(stride) - 1;
+  // Position offset k of this row looks at; false if there is none (off the grid, out of range, the row itself).
+  auto target = [&](int k, int& x, int& y, int& z) -> bool {
+    const int a = k / (K * K), b = (k / K) % K, cc = k % K;
+    if (MODE == 0) {
+      x = c.y + dil * (a - r); y = c.z + dil * (b - r); z = c.w + dil * (cc - r);
+      return usable && !(a == r && b == r && cc == r) && in_range(x) && in_range(y) && in_range(z);
+    }
+    const int nx = c.y + pad - dil * a, ny = c.z + pad - dil * b, nz = c.w + pad - dil * cc;
+    const bool on_grid = pow2 ? (((nx | ny | nz) & (stride - 1)) == 0) : (nx % stride == 0 && ny % stride == 0 && nz % stride == 0);
+    x = pow2 ? nx >> shift : nx / stride; y = pow2 ? ny >> shift : ny / stride; z = pow2 ? nz >> shift : nz / stride;
+    return usable && nx >= 0 && ny >= 0 && nz >= 0 && on_grid && in_range(x) && in_range(y) && in_range(z);
+  };
+  // 1. candidates: offsets whose position the occupancy filter does not rule out (all reads in flight together)
+  uint32_t cand = 0u;
+  {
+    uint32_t word[KV];
+#pragma unroll
+    for (int k = 0; k < KV; ++k) {
+      int x, y, z;
+      const bool valid = target(k, x, y, z);
+      word[k] = 0xFFFFFFFFu;
+      if (valid) word[k] = occ != nullptr ? __ldg(occ + occ_word(c.x, x, y, z)) : 0u;
+      word[k] = (word[k] >> (z & 31)) & 1u;   // 1: ruled out
+      s_v[k][tid] = (MODE == 0 && k == (r * K + r) * K + r && live) ? j : -1;
+    }
+#pragma unroll
+    for (int k = 0; k < KV; ++k) cand |= (word[k] ^ 1u) << k;
+  }
+  // 2. the candidates' table lookups, four at a time
+  while (cand != 0u) {
+#ifndef SPCONV_PROBE_BATCH
+#define SPCONV_PROBE_BATCH 4
+#endif
+    constexpr int B = SPCONV_PROBE_BATCH;
+    int kk[B];
+    uint64_t key[B];
+    LocSlot got[B];
+    uint32_t slot[B];
+#pragma unroll
+    for (int u = 0; u < B; ++u) {
+      kk[u] = -1;
+      key[u] = kEmptyKey; got[u].key = kEmptyKey; got[u].row = -1; slot[u] = 0u;
+      if (cand != 0u) {
+        kk[u] = __ffs(int(cand)) - 1;
+        cand &= cand - 1u;
+        int x, y, z;
+        target(kk[u], x, y, z);
+        key[u] = pack_key(c.x, x, y, z);
+        slot[u] = hash_key(key[u]) & capmask;
+        got[u] = load_slot(table, slot[u]);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < B; ++u) {
+      if (kk[u] < 0) continue;
+      LocSlot g = got[u];
+      for (uint32_t probe = 0; probe <= capmask; ++probe) {
+        if (g.key == key[u]) { s_v[kk[u]][tid] = g.row; break; }
+        if (g.key == kEmptyKey) break;
+        slot[u] = (slot[u] + 1) & capmask;
+        g = load_slot(table, slot[u]);
+      }
+    }
+  }
+  // 3. the row's entries leave in both layouts, with the row's offset set and the block's hit counts
+  uint32_t mask = 0u;
+  int v[KV];
+#pragma unroll
+  for (int k = 0; k < KV; ++k) {
+    v[k] = s_v[k][tid];
+    const bool present = v[k] >= 0;
+    mask |= present ? (1u << k) : 0u;
+    if (live) nbr[size_t(k) * nq + j] = v[k];
+    const unsigned ballot = __ballot_sync(0xffffffffu, present);
+    if (lane == 0 && ballot != 0u) atomicAdd(&s_cnt[k], unsigned(__popc(ballot)));
+  }
+  if (live) row_mask[j] = mask;
+  // Row-major copy: the warp writes its 32 rows together, eight lanes per row (16 bytes each), so that a store
+  // instruction covers four whole rows instead of touching 32 (the entries come back from shared memory).
+  __syncwarp();
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int q = lane & 7, rt = (tid & ~31) + 4 * i + (lane >> 3);
+    const int jr = blockIdx.x * kBlock + rt;
+    if (jr < nq && 4 * q < KV) {
+      int4 t;
+      t.x = s_v[4 * q][rt];
+      t.y = 4 * q + 1 < KV ? s_v[4 * q + 1 < KV ? 4 * q + 1 : 0][rt] : -1;
+      t.z = 4 * q + 2 < KV ? s_v[4 * q + 2 < KV ? 4 * q + 2 : 0][rt] : -1;
+      t.w = 4 * q + 3 < KV ? s_v[4 * q + 3 < KV ? 4 * q + 3 : 0][rt] : -1;
+      reinterpret_cast<int4*>(nbr_rows + size_t(jr) * 32)[q] = t;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < KV) {
+    const unsigned cnt = s_cnt[threadIdx.x];
+    blockcnt[size_t(threadIdx.x) * gridDim.x + blockIdx.x] = int32_t(cnt);
+    if (offset_cnt != nullptr && cnt != 0u) atomicAdd(&offset_cnt[threadIdx.x], cnt);
+  }
+  SPCONV_TL(3);
+}
+
+// Inverse convolution, any kernel volume: one offset per thread, grid = (ceil(nq/256), kvol); same outputs as
+// k_subm_probe (offset-major table and per-block hit counts).
+__global__ void k_inverse_probe(const int4* __restrict__ qcoords, int nq, int K, int stride, int dil, const LocSlot* __restrict__ table,
+                                uint32_t capmask, int32_t* __restrict__ nbr,
+                                int32_t* __restrict__ blockcnt, unsigned* __restrict__ offset_cnt, uint32_t* __restrict__ status,
+                                const __grid_constant__ OffsetIndex index) {
+  chain_begin();
+  const int k = blockIdx.y;
   const int j = blockIdx.x * kBlock + threadIdx.x;
   int ia, ib, ic;
-  offset_index(index, k0, KZ, ia, ib, ic);
-  const int dx = dil * (ia - r), dy = dil * (ib - r);
-  const bool live = j < n;
-  int4 c = make_int4(0, 0, 0, 0);
-  if (live) c = coords[j];
-  const int x = c.y + dx, y = c.z + dy;
-  const bool xy_ok = live && in_range(x) && in_range(y);
-  uint64_t key[KZ], got[KZ];
-  uint32_t slot[KZ];
-  int v[KZ];
-#pragma unroll
-  for (int u = 0; u < KZ; ++u) {
-    const int z = c.w + dil * (u - r);
-    const bool self = (dx | dy) == 0 && u == r;
-    const bool valid = xy_ok && in_range(z) && !self;
-    key[u] = valid ? pack_key(c.x, x, y, z) : kEmptyKey;   // an empty key never matches: a miss below
-    slot[u] = hash_key(key[u]) & capmask;
-    got[u] = valid ? __ldg(keys + slot[u]) : kEmptyKey;
-    v[u] = (self && live) ? j : -1;
-  }
-#pragma unroll
-  for (int u = 0; u < KZ; ++u) {
-    if (key[u] == kEmptyKey) continue;
-    uint64_t g = got[u];
-    uint32_t sl = slot[u];
-    for (uint32_t probe = 0; probe <= capmask; ++probe) {
-      if (g == key[u]) { v[u] = __ldg(vals + sl); break; }
-      if (g == kEmptyKey) break;
-      sl = (sl + 1) & capmask;
-      g = __ldg(keys + sl);
+  offset_index(index, k, K, ia, ib, ic);
+  const int pad = dil * ((K - 1) / 2);
+  int v = -1;
+  if (j < nq) {
+    const int4 c = qcoords[j];
+    if (!(in_range(c.x) && in_range(c.y) && in_range(c.z) && in_range(c.w))) {
+      if (k == 0) atomicOr(status, kDevCoordRange);
+    } else {
+      const int nx = c.y + pad - dil * ia, ny = c.z + pad - dil * ib, nz = c.w + pad - dil * ic;
+      if (nx >= 0 && ny >= 0 && nz >= 0 && nx % stride == 0 && ny % stride == 0 && nz % stride == 0) {
+        const int x = nx / stride, y = ny / stride, z = nz / stride;
+        if (in_range(x) && in_range(y) && in_range(z)) v = table_find(table, capmask, pack_key(c.x, x, y, z));
+      }
     }
+    nbr[size_t(k) * nq + j] = v;
   }
-#pragma unroll
-  for (int u = 0; u < KZ; ++u) {
-    const int k = k0 + u;
-    if (live) nbr[size_t(k) * n + j] = v[u];
-    const int cnt = __syncthreads_count(v[u] >= 0);
-    if (threadIdx.x == 0) {
-      blockcnt[size_t(k) * gridDim.x + blockIdx.x] = cnt;
-      if (offset_cnt != nullptr && cnt != 0) atomicAdd(&offset_cnt[k], unsigned(cnt));
-    }
+  const int cnt = __syncthreads_count(v >= 0);
+  if (threadIdx.x == 0) {
+    blockcnt[size_t(k) * gridDim.x + blockIdx.x] = cnt;
+    if (offset_cnt != nullptr && cnt != 0) atomicAdd(&offset_cnt[k], unsigned(cnt));
   }
 }
 
@@ -270,6 +427,7 @@ __global__ void k_scan_counts(const int32_t* __restrict__ cnt, int64_t M, int64_
                               int kvol, int64_t* __restrict__ offset_start, int64_t* __restrict__ total_out,
                               int8_t* __restrict__ bitpos) {
   chain_begin();
+  SPCONV_TL(10);
   scan_counts_block<1024>(cnt, M, excl, nblk, kvol, offset_start, total_out, bitpos);
 }
 
@@ -287,20 +445,38 @@ __device__ __forceinline__ int block_rank(bool flag) {
 }
 
 // Per-offset (input, output) pairs from the offset table: stream compaction of nbr[k][:].
+// The first list position of block (x, k) is either read from a scan of all blocks' hit counts (excl) or, with
+// excl == nullptr, summed by the block itself from the probe kernel's counts: the totals of the offsets before k
+// (offset_cnt) plus the hits of the blocks before x within offset k (blockcnt[k][0 .. x)).
 __global__ void k_subm_emit(const int32_t* __restrict__ nbr, int n, const int64_t* __restrict__ excl,
+                            const int32_t* __restrict__ blockcnt, const unsigned* __restrict__ offset_cnt,
                             int32_t* __restrict__ pair_in, int32_t* __restrict__ pair_out, int64_t capacity) {
   chain_begin();
+  SPCONV_TL(8);
+  __shared__ long long base_s;
   const int k = blockIdx.y;
   const int j = blockIdx.x * kBlock + threadIdx.x;
   const int v = j < n ? nbr[size_t(k) * n + j] : -1;
+  if (excl == nullptr) {
+    long long part = 0;
+    for (int b = threadIdx.x; b < int(blockIdx.x); b += kBlock) part += blockcnt[size_t(k) * gridDim.x + b];
+    if (int(threadIdx.x) < k) part += (long long)offset_cnt[threadIdx.x];
+    if (threadIdx.x == 0) base_s = 0;
+    __syncthreads();
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) part += __shfl_down_sync(0xffffffffu, part, off);
+    if ((threadIdx.x & 31) == 0 && part != 0) atomicAdd(reinterpret_cast<unsigned long long*>(&base_s), (unsigned long long)part);
+    __syncthreads();
+  }
   const int rank = block_rank(v >= 0);
   if (v >= 0) {
-    const int64_t p = excl[size_t(k) * gridDim.x + blockIdx.x] + rank;
+    const int64_t p = (excl != nullptr ? excl[size_t(k) * gridDim.x + blockIdx.x] : int64_t(base_s)) + rank;
     if (p < capacity) {   // the lists may have been sized from an estimate (the host then repeats the emission)
       pair_in[p] = v;
       pair_out[p] = j;
     }
   }
+  SPCONV_TL(9);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -327,7 +503,7 @@ __global__ void k_strided_candidates(const int4* __restrict__ coords, int n, int
       const int ox = pow2 ? nx >> shift : nx / s, oy = pow2 ? ny >> shift : ny / s, oz = pow2 ? nz >> shift : nz / s;
       if (in_range(ox) && in_range(oy) && in_range(oz) && in_range(c.x)) {
         bool present;
-        slot = table_insert(keys2, capmask2, pack_key(c.x, ox, oy, oz), &present);
+        slot = table_insert<1>(keys2, capmask2, pack_key(c.x, ox, oy, oz), &present);
         if (slot < 0) atomicOr(status, kDevTableFull);
         else atomicMin(owner_cid + slot, k * n + i);   // the smallest candidate id owns the cell
       } else {
@@ -379,7 +555,7 @@ __global__ void k_owner_assign(const int32_t* __restrict__ cand_slot, const int3
 // Offset table and pair lists of the strided map (second stage of the paper's two-stage table).
 __global__ void k_strided_emit(const int32_t* __restrict__ cand_slot, const int32_t* __restrict__ slot_out, int n,
                                int64_t n_out, const int64_t* __restrict__ excl, int32_t* __restrict__ nbr,
-                               int32_t* __restrict__ pair_in, int32_t* __restrict__ pair_out) {
+                               int32_t* __restrict__ pair_in, int32_t* __restrict__ pair_out, int32_t* __restrict__ nbr_rows) {
   chain_begin();
   const int k = blockIdx.y;
   const int i = blockIdx.x * kBlock + threadIdx.x;
@@ -388,6 +564,7 @@ __global__ void k_strided_emit(const int32_t* __restrict__ cand_slot, const int3
   if (slot >= 0) {
     const int o = slot_out[slot];
     nbr[size_t(k) * n_out + o] = i;
+    if (nbr_rows != nullptr) nbr_rows[size_t(o) * 32 + k] = i;   // the row-major copy the tile plan reads
     const int64_t p = excl[size_t(k) * gridDim.x + blockIdx.x] + rank;
     pair_in[p] = i;
     pair_out[p] = o;
@@ -401,10 +578,11 @@ __global__ void k_strided_emit(const int32_t* __restrict__ cand_slot, const int3
 // full or absent and the kernel skips the absent ones.
 // Row keys of the tile plan; also marks the unused rows of the last tile (tile_rows beyond n_out) with -1.
 __global__ void k_row_keys(const int32_t* __restrict__ nbr, int64_t n_out, int64_t n_padded, int kvol,
-                           const int8_t* __restrict__ bitpos, uint32_t* __restrict__ keys, int32_t* __restrict__ rows,
-                           int32_t* __restrict__ tile_rows) {
+                           const int8_t* __restrict__ bitpos, const unsigned* __restrict__ offset_cnt, uint32_t* __restrict__ keys,
+                           int32_t* __restrict__ rows, int32_t* __restrict__ tile_rows) {
   __shared__ int8_t pos[32];
-  if (threadIdx.x < 32) pos[threadIdx.x] = threadIdx.x < kvol ? bitpos[threadIdx.x] : int8_t(0);
+  if (threadIdx.x < 32)
+    pos[threadIdx.x] = int(threadIdx.x) >= kvol ? int8_t(0) : (offset_cnt != nullptr ? int8_t(offset_rank(int(threadIdx.x), kvol, nullptr, nullptr, offset_cnt)) : bitpos[threadIdx.x]);
   __syncthreads();
   const int64_t o = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
   if (o >= n_out) {
@@ -434,12 +612,14 @@ constexpr int kSortThreads = 256, kSortItemsSmall = 4, kSortItemsLarge = 8, kSor
 
 template <int kSortItems>
 __global__ void __launch_bounds__(kSortThreads)
-k_sort_rows_coop(const int32_t* __restrict__ nbr, int64_t n_out, int64_t n_padded, int kvol, const int8_t* __restrict__ bitpos,
+k_sort_rows_coop(const int32_t* __restrict__ nbr, const int32_t* __restrict__ nbr_rows, const uint32_t* __restrict__ row_mask,
+                 int64_t n_out, int64_t n_padded, int kvol, const int8_t* __restrict__ bitpos,
                  const unsigned* __restrict__ offset_cnt, int begin_bit, uint32_t* __restrict__ keys_a, int32_t* __restrict__ rows_a,
                  uint32_t* __restrict__ keys_b, int32_t* __restrict__ rows_b, uint32_t* __restrict__ block_hist /* [gridDim.x][256] */,
                  int32_t* __restrict__ tile_rows, const int32_t* __restrict__ scan_cnt, int64_t scan_m, int64_t* __restrict__ scan_excl,
                  int scan_nblk, int64_t* __restrict__ scan_offset_start, int64_t* __restrict__ scan_total) {
   chain_begin();
+  SPCONV_TL(4);
   namespace cg = cooperative_groups;
   cg::grid_group grid = cg::this_grid();
   constexpr int kSortTile = kSortThreads * kSortItems;
@@ -465,8 +645,22 @@ k_sort_rows_coop(const int32_t* __restrict__ nbr, int64_t n_out, int64_t n_padde
     const int64_t o = base + r * 32;
     uint32_t m = 0;
     if (o < n_out) {
-      for (int k = 0; k < kvol; ++k)
-        if (nbr[size_t(k) * n_out + o] >= 0) m |= 1u << pos[k];
+      // The row's offset set: ready-made (row_mask), from its row of the row-major table, or from the offset-major one.
+      uint32_t raw = 0u;
+      if (row_mask != nullptr) {
+        raw = row_mask[o];
+      } else if (nbr_rows != nullptr) {
+        const int4* rp = reinterpret_cast<const int4*>(nbr_rows + size_t(o) * 32);
+        for (int q = 0; 4 * q < kvol; ++q) {
+          const int4 t = __ldcg(rp + q);
+          raw |= (t.x >= 0 ? 1u : 0u) << (4 * q) | (t.y >= 0 ? 2u : 0u) << (4 * q) | (t.z >= 0 ? 4u : 0u) << (4 * q) | (t.w >= 0 ? 8u : 0u) << (4 * q);
+        }
+        raw &= kvol >= 32 ? 0xFFFFFFFFu : ((1u << kvol) - 1u);
+      } else {
+        for (int k = 0; k < kvol; ++k)
+          if (nbr[size_t(k) * n_out + o] >= 0) raw |= 1u << k;
+      }
+      for (int k = 0; k < kvol; ++k) m |= ((raw >> k) & 1u) << pos[k];
       // Gray -> binary: consecutive keys differ in one offset where possible.
       m ^= m >> 1; m ^= m >> 2; m ^= m >> 4; m ^= m >> 8; m ^= m >> 16;
     } else if (o < n_padded) {
@@ -503,25 +697,39 @@ k_sort_rows_coop(const int32_t* __restrict__ nbr, int64_t n_out, int64_t n_padde
       block_hist[size_t(blockIdx.x) * 256 + tid] = run;
     }
     grid.sync();
-    {  // per digit: items of earlier blocks with this digit, and of all blocks.  Warp w sums the blocks
-       // b = w (mod 8), each lane eight digits, so that a thread has eight independent loads in flight.
+    {  // per digit: items of earlier blocks with this digit, and of all blocks.  Warp w sums the blocks b = w (mod 8);
+       // a lane takes eight consecutive digits of a block's counts as two vector loads, and the loads of up to
+       // twelve blocks are in flight together (one round trip for grids of up to 96 blocks).
       before_s[tid] = 0u; total_s[tid] = 0u;
       __syncthreads();
       uint32_t bef[8], tot[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) { bef[j] = 0u; tot[j] = 0u; }
-#pragma unroll 2
-      for (unsigned b = warp; b < gridDim.x; b += kSortThreads / 32) {
-        const uint32_t* hrow = block_hist + size_t(b) * 256 + lane;
-        const bool earlier = b < blockIdx.x;
+      constexpr int kBatch = 12;
+      for (unsigned b0 = warp; b0 < gridDim.x; b0 += kBatch * (kSortThreads / 32)) {
+        uint4 c[kBatch][2];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { const uint32_t c = hrow[32 * j]; tot[j] += c; if (earlier) bef[j] += c; }
+        for (int u = 0; u < kBatch; ++u) {   // (volatile: the loads are issued back to back, ahead of the sums)
+          const unsigned b = b0 + u * (kSortThreads / 32);
+          const uint4* src = reinterpret_cast<const uint4*>(block_hist + size_t(b < gridDim.x ? b : b0) * 256 + lane * 8);
+          asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(c[u][0].x), "=r"(c[u][0].y), "=r"(c[u][0].z), "=r"(c[u][0].w) : "l"(src));
+          asm volatile("ld.global.cg.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(c[u][1].x), "=r"(c[u][1].y), "=r"(c[u][1].z), "=r"(c[u][1].w) : "l"(src + 1));
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const unsigned b = b0 + u * (kSortThreads / 32);
+          if (b >= gridDim.x) continue;
+          const bool earlier = b < blockIdx.x;
+          const uint32_t vals8[8] = {c[u][0].x, c[u][0].y, c[u][0].z, c[u][0].w, c[u][1].x, c[u][1].y, c[u][1].z, c[u][1].w};
+#pragma unroll
+          for (int j = 0; j < 8; ++j) { tot[j] += vals8[j]; if (earlier) bef[j] += vals8[j]; }
+        }
       }
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { atomicAdd(&before_s[lane + 32 * j], bef[j]); atomicAdd(&total_s[lane + 32 * j], tot[j]); }
+      for (int j = 0; j < 8; ++j) { atomicAdd(&before_s[lane * 8 + j], bef[j]); atomicAdd(&total_s[lane * 8 + j], tot[j]); }
       __syncthreads();
-      // digit tid: exclusive prefix of the totals over all smaller digits
       const uint32_t before = before_s[tid], total = total_s[tid];
+      // digit tid: exclusive prefix of the totals over all smaller digits
       uint32_t incl = total;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) { const uint32_t t = __shfl_up_sync(0xffffffffu, incl, off); if (lane >= off) incl += t; }
@@ -543,7 +751,7 @@ k_sort_rows_coop(const int32_t* __restrict__ nbr, int64_t n_out, int64_t n_padde
       if (!last) kout[at] = key[r];
       rout[at] = row[r];
     }
-    if (last) break;
+    if (last) { SPCONV_TL(5); break; }
     grid.sync();
 #pragma unroll
     for (int r = 0; r < kSortItems; ++r) {
@@ -554,6 +762,8 @@ k_sort_rows_coop(const int32_t* __restrict__ nbr, int64_t n_out, int64_t n_padde
     __syncthreads();   // warp_hist and goff are rewritten by the next pass
   }
 }
+
+
 
 __global__ void k_iota_rows(int32_t* rows, int64_t n_out, int64_t n_padded) {
   const int64_t o = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -672,6 +882,107 @@ __global__ void k_tile_plan(const int32_t* __restrict__ tile_rows, const int32_t
     // the build a copy and a stream synchronisation.
     if (host_totals != nullptr) {
       for (int i = threadIdx.x; i < totals_words; i += blockDim.x) host_totals[i] = __ldcg(totals + i);
+      __threadfence_system();
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        *reinterpret_cast<volatile int64_t*>(host_totals + totals_words) = 1;
+        __threadfence_system();
+      }
+    }
+  }
+}
+
+
+// The same plan from the row-major table (kernel volumes up to 32): thread (warp w, lane k) takes offset k of the
+// tile rows 32w .. 32w + 31.  A row of the table is one 128-byte line, so the 32 loads of a thread are 32
+// coalesced warp loads, all in flight together, where the offset-major table costs a 32-byte sector per entry.
+// The compacted lists are put together in shared memory and leave as whole lines.
+constexpr int kPlanNbrPitch = kTileRows + 4;    // ints per offset in shared memory (16-byte aligned rows, banks skewed by 4)
+constexpr int kPlanCrowPitch = kTileRows + 16;  // bytes per offset
+__global__ void __launch_bounds__(kTileRows)
+k_tile_plan_rows(const int32_t* __restrict__ tile_rows, const int32_t* __restrict__ nbr_rows, int kvol,
+                 int32_t* __restrict__ tile_nbr, uint8_t* __restrict__ tile_crow, uint32_t* __restrict__ tile_mask,
+                 uint32_t* __restrict__ tile_absent, unsigned long long* __restrict__ block_counter,
+                 unsigned* __restrict__ tiles_done, int32_t* __restrict__ sorted_tiles, uint32_t* __restrict__ status_words,
+                 const int64_t* __restrict__ totals, int totals_words, int64_t* __restrict__ host_totals, int report_from_counts) {
+  chain_begin();
+  SPCONV_TL(6);
+  __shared__ __align__(16) int32_t s_nbr[32][kPlanNbrPitch];
+  __shared__ __align__(16) uint8_t s_crow[32][kPlanCrowPitch];
+  __shared__ int s_cnt[32][kTileRows / 32];
+  __shared__ bool last_block;
+  const int t = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int my_row = tile_rows[size_t(t) * kTileRows + tid];
+  int v[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const int row = __shfl_sync(0xffffffffu, my_row, i);
+    v[i] = (row >= 0 && lane < kvol) ? __ldcg(nbr_rows + size_t(row) * 32 + lane) : -1;
+  }
+  uint32_t pm = 0u;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) pm |= (v[i] >= 0 ? 1u : 0u) << i;
+  s_cnt[lane][warp] = __popc(pm);
+  if (lane < kvol) tile_absent[(size_t(t) * kvol + lane) * 4 + warp] = ~pm;   // rows of this warp's 32 without an input
+  __syncthreads();
+  int base = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < kTileRows / 32; ++w) { const int c = s_cnt[lane][w]; if (w < warp) base += c; total += c; }
+  {  // this thread's entries of offset `lane`, in row order, behind those of the warps before it
+    int at = base;
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if ((pm >> i) & 1u) { s_nbr[lane][at] = v[i]; s_crow[lane][at] = uint8_t(32 * warp + i); ++at; }
+  }
+  // entries past an offset's count: no row
+  for (int k = 0; k < kvol; ++k) {
+    int tk = 0;
+#pragma unroll
+    for (int w = 0; w < kTileRows / 32; ++w) tk += s_cnt[k][w];
+    if (tid >= tk) { s_nbr[k][tid] = -1; s_crow[k][tid] = 0; }
+  }
+  const unsigned word = __ballot_sync(0xffffffffu, lane < kvol && total > 0);
+  __syncthreads();
+  {
+    int4* dst = reinterpret_cast<int4*>(tile_nbr + size_t(t) * kvol * kTileRows);
+    for (int i = tid; i < kvol * (kTileRows / 4); i += kTileRows) {
+      const int k = i / (kTileRows / 4), q = i % (kTileRows / 4);
+      dst[i] = *reinterpret_cast<const int4*>(&s_nbr[k][4 * q]);
+    }
+    int4* dstc = reinterpret_cast<int4*>(tile_crow + size_t(t) * kvol * kTileRows);
+    for (int i = tid; i < kvol * (kTileRows / 16); i += kTileRows) {
+      const int k = i / (kTileRows / 16), q = i % (kTileRows / 16);
+      dstc[i] = *reinterpret_cast<const int4*>(&s_crow[k][16 * q]);
+    }
+  }
+  if (tid == 0) {
+    tile_mask[t] = word;
+    atomicAdd(block_counter, (unsigned long long)__popc(word));
+  }
+  // The block that finishes last orders the tiles for the forward's schedule and reports to the host (see k_tile_plan).
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) last_block = atomicAdd(tiles_done, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (last_block) {
+    __threadfence();
+    schedule_tiles_block(tile_mask, int(gridDim.x), 1, kvol, sorted_tiles, status_words);
+    if (host_totals != nullptr) {
+      for (int i = threadIdx.x; i < totals_words; i += blockDim.x) host_totals[i] = __ldcg(totals + i);
+#ifdef SPCONV_KMAP_TIMELINE
+      if (threadIdx.x == 0) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); SPCONV_TL_RAW(7, t); }
+#endif
+      if (report_from_counts) {
+        // pair count and offset starts straight from the probe's per-offset totals (the words behind the totals block)
+        __syncthreads();
+        if (threadIdx.x == 0) {
+          const unsigned* cnt = reinterpret_cast<const unsigned*>(totals + totals_words);
+          int64_t run = 0;
+          for (int k = 0; k < kvol; ++k) { host_totals[8 + k] = run; run += int64_t(__ldcg(cnt + k)); }
+          host_totals[8 + kvol] = run;
+          host_totals[1] = run;
+        }
+      }
       __threadfence_system();
       __syncthreads();
       if (threadIdx.x == 0) {
@@ -876,6 +1187,7 @@ int coop_sort_capacity(int device) {
   return cap[device];
 }
 
+
 // Largest number of offsets along one axis through which a single input position can reach an output cell.
 int max_candidates_per_axis(int K, int s, int d) {
   int best = 0;
@@ -916,10 +1228,33 @@ struct StageTimer {
 struct StageTimer { explicit StageTimer(cudaStream_t) {} };
 #define SPCONV_STAGE(t, what)
 #endif
+#ifdef SPCONV_KMAP_TIMELINE
+struct TimelineDump {
+  cudaStream_t stream;
+  std::chrono::steady_clock::time_point h0 = std::chrono::steady_clock::now();
+  double hs[16]; const char* hn[16]; int nh = 0;
+  void host(const char* what) { if (nh < 16) { hs[nh] = std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - h0).count(); hn[nh++] = what; } }
+  ~TimelineDump() {
+    for (int i = 0; i < nh; ++i) std::fprintf(stderr, "  host %-16s %8.2f us\n", hn[i], hs[i]);
+    cudaDeviceSynchronize();
+    unsigned long long t[32];
+    if (cudaMemcpyFromSymbol(t, g_kmap_timeline, sizeof(t)) != cudaSuccess) return;
+    const char* names[] = {"insert start", "insert end(b0)", "probe start", "probe end(b0)", "sort start", "sort end(b0)", "plan start", "plan report", "emit start", "emit end(b0)", "scan start"};
+    for (int i = 0; i < 11; ++i) std::fprintf(stderr, "  tl %-16s %8.2f us\n", names[i], (double(t[i]) - double(t[0])) * 1e-3);
+  }
+};
+#endif
 
 int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, int kernel, int submanifold,
-                    cudaStream_t stream, spconv_kmap** out, const std::function<int(spconv_kmap*)>* before_wait) {
+                    cudaStream_t stream, spconv_kmap** out, const std::function<int(spconv_kmap*)>* before_wait,
+                    const int32_t* fine_coords, int64_t n_fine) {
   [[maybe_unused]] StageTimer stages(stream);
+#ifdef SPCONV_KMAP_TIMELINE
+  TimelineDump timeline_dump{stream};
+#define SPCONV_HOST_TL(what) timeline_dump.host(what)
+#else
+#define SPCONV_HOST_TL(what)
+#endif
   SPCONV_STAGE(stages, "start");
   const int K = kernel, s = stride, d = dilation;
   const int kvol = K * K * K;
@@ -927,24 +1262,35 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   if (!km) return SPCONV_ERR_ALLOC;
   struct Guard { spconv_kmap* km; ~Guard() { if (km) destroy_kmap_impl(km); } } guard{km};
   km->kernel = K; km->stride = s; km->dilation = d; km->submanifold = submanifold; km->kvol = kvol;
+  // Inverse convolution (fine_coords given): the location table is built over `coords` (the coarse positions, the
+  // rows of the input features) and probed from the fine positions, which are the output rows.  Like a submanifold
+  // map its output rows are known up front, so both take the same path below with nq query rows.
+  const bool inverse = fine_coords != nullptr;
+  const bool known_outputs = submanifold || inverse;
+  const int64_t nq = inverse ? n_fine : n;
+  km->inverse = inverse ? 1 : 0;
   km->n_in = n;
   km->stream = stream;
   km->mask_words = (kvol + 31) / 32;
   km->offset_start.assign(size_t(kvol) + 1, 0);
   SPCONV_CUDA_TRY(cudaGetDevice(&km->device));
-  if (n == 0) {  // empty map: no device memory at all
+  if (nq == 0 || (n == 0 && !inverse)) {  // empty map: no device memory at all
     *out = km; guard.km = nullptr;
     return SPCONV_OK;
   }
 
-  const int nblk = int((n + kBlock - 1) / kBlock);
+  const int nblk = int((nq + kBlock - 1) / kBlock);
   const int64_t M = int64_t(nblk) * kvol;
   // Load factor of the location table: at most 1/kTableSlack.  Probe sequences are walked by whole warps (a warp
   // takes as many rounds as its unluckiest lane), so short sequences matter more than the table's size.
   static const int kTableSlack = [] { const char* e = std::getenv("SPCONV_KMAP_TABLE_SLACK"); return e != nullptr ? std::max(2, std::atoi(e)) : 4; }();
-  const uint32_t cap1 = pow2_at_least(uint64_t(kTableSlack) * n);
+  const uint32_t cap1 = pow2_at_least(uint64_t(kTableSlack) * std::max<int64_t>(n, 1));
   const dim3 grid_kn(nblk, kvol);
   const int4* coords4 = reinterpret_cast<const int4*>(coords);
+  const int4* qcoords4 = inverse ? reinterpret_cast<const int4*>(fine_coords) : coords4;
+  const int nblk_in = int((n + kBlock - 1) / kBlock);   // blocks over the rows that go into the location table
+  // Kernel volumes up to 32 keep a second, row-major copy of the offset table (rows of 32 entries) for the tile plan.
+  const bool rows_table = kvol <= 32;
 
   keep_pool_cached(km->device);
   PinnedHost host;
@@ -957,7 +1303,7 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   // ----- scratch arena (freed stream-ordered when this function leaves)
   uint32_t cap2 = 0;
   int64_t n_out_max = n;
-  if (!submanifold) {
+  if (!known_outputs) {
     const int cpa = max_candidates_per_axis(K, s, d);
     n_out_max = std::min<int64_t>(n * int64_t(cpa) * cpa * cpa, int64_t(2000000000));
     cap2 = pow2_at_least(uint64_t(2) * n_out_max);
@@ -971,20 +1317,23 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     if (!plan_sorted) return size_t(0);
     cub::DeviceRadixSort::SortPairs(nullptr, *cub_bytes, static_cast<uint32_t*>(nullptr), static_cast<uint32_t*>(nullptr),
                                     static_cast<int32_t*>(nullptr), static_cast<int32_t*>(nullptr), int(items), sort_begin_bit, kvol, stream);
-    return pad256(*cub_bytes) + pad256(size_t(items) * 4) * 4 + pad256((size_t(items) / (kSortThreads * kSortItemsSmall) + 3) * 1024) + 1024;
+    return pad256(*cub_bytes) + pad256(size_t(items) * 4) * 4 + pad256((size_t(items) / (kSortThreads * kSortItemsSmall) + 8) * 1024) + 1024;
   };
   size_t cub_bytes = 0;
-  size_t scratch_bytes = pad256(size_t(cap1) * 8) + pad256(size_t(cap1) * 4) + pad256(size_t(M) * 4) * 2 +
+  size_t scratch_bytes = pad256(size_t(cap1) * sizeof(LocSlot)) + pad256(size_t(kOccWords) * 4) + pad256(size_t(M) * 4) * 2 +
                          pad256(size_t(M) * 8) * 2 + pad256((size_t(kvol) + 1 + 8 + 16) * 8) + pad256(32) + 4096;
-  if (submanifold) scratch_bytes += sort_bytes_for(n, &cub_bytes);   // n_out = n: the sort's buffers ride along
-  if (!submanifold)
+  if (known_outputs) scratch_bytes += sort_bytes_for(nq, &cub_bytes);   // n_out is known: the sort's buffers ride along
+  if (known_outputs && rows_table) scratch_bytes += pad256(size_t(nq) * 128) + pad256(size_t(nq) * 4);
+  if (!known_outputs)
     scratch_bytes += pad256(size_t(cap2) * 8) + pad256(size_t(cap2) * 4) * 2 + pad256(size_t(kvol) * n * 4);
   Scratch scratch;
   scratch.stream = stream;
   SPCONV_CUDA_TRY(cudaMallocAsync(&scratch.ptr, scratch_bytes, stream));
   Arena sa{static_cast<char*>(scratch.ptr), scratch_bytes, 0};
-  uint64_t* keys1 = sa.take<uint64_t>(cap1);
-  int32_t* vals1 = sa.take<int32_t>(cap1);
+  LocSlot* table1 = sa.take<LocSlot>(cap1);
+  // the occupancy filter lies right behind the table: one fill empties both
+  uint32_t* occ = (known_outputs && rows_table) ? sa.take<uint32_t>(kOccWords) : nullptr;
+  const size_t table_fill_bytes = occ != nullptr ? size_t(reinterpret_cast<char*>(occ + kOccWords) - reinterpret_cast<char*>(table1)) : size_t(cap1) * sizeof(LocSlot);
   int32_t* cnt_a = sa.take<int32_t>(M);
   int32_t* cnt_b = sa.take<int32_t>(M);
   int64_t* excl_a = sa.take<int64_t>(M);
@@ -1000,7 +1349,13 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   unsigned long long* d_tile_blocks = reinterpret_cast<unsigned long long*>(d_totals + 3);
   unsigned* d_tiles_done = reinterpret_cast<unsigned*>(d_totals + 4);
   uint64_t* keys2 = nullptr; int32_t* owner_cid = nullptr; int32_t* slot_out = nullptr; int32_t* cand_slot = nullptr;
-  if (!submanifold) {
+  int32_t* nbr_rows = nullptr;     // [n_out][32] row-major offset table (scratch)
+  uint32_t* row_mask = nullptr;    // [n_out] offset set of every row, when the probe kernel forms it
+  if (known_outputs && rows_table) {
+    nbr_rows = sa.take<int32_t>(size_t(nq) * 32);
+    row_mask = sa.take<uint32_t>(size_t(nq));
+  }
+  if (!known_outputs) {
     keys2 = sa.take<uint64_t>(cap2);
     owner_cid = sa.take<int32_t>(cap2);
     slot_out = sa.take<int32_t>(cap2);
@@ -1034,6 +1389,12 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   // nbr, the per-offset counts' bit order (d_bitpos, written by k_scan_counts) and sort buffers.
   int64_t* flag_target = nullptr;   // pinned host buffer the tile plan's last block reports into (submanifold path)
   std::function<int()> after_sort;   // (submanifold path) enqueues the pair emission beside the tile plan
+  // Maps whose outputs are known up front and whose kernel volume fits the 32 per-offset counters need no scan of the
+  // probe's per-block counts: the report to the host and the bit order of the sort come from the per-offset totals,
+  // and the emission's blocks sum their own list positions.
+  const bool counts_based = known_outputs && d_offset_cnt != nullptr;
+  const int32_t* plan_rows = nullptr;      // row-major offset table the sort and the tile plan read, when there is one
+  const uint32_t* plan_row_mask = nullptr; // offset sets of the rows, when the probe kernel has formed them
   auto enqueue_tile_plan = [&](Arena& ta, size_t cub_tmp_bytes, bool scan_pending) -> int {
     const int64_t no = km->n_out, padded = int64_t(km->n_tiles) * kTileRows;
     const int rb = int((padded + kBlock - 1) / kBlock);
@@ -1049,13 +1410,16 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
       uint32_t* block_hist = ta.take<uint32_t>(size_t(sort_blocks + 1) * 256);
       void* cub_tmp = ta.take<char>(cub_tmp_bytes);
       size_t tmp_bytes = cub_tmp_bytes;
+      const unsigned* order_cnt = (scan_pending || counts_based) ? d_offset_cnt : nullptr;   // the probe's per-offset totals order the key bits
       if (sort_blocks + 1 <= coop_sort_capacity(km->device)) {
         // every block resident at once: keys and all sort passes in one cooperative launch
         const int32_t* nbr_arg = km->d.nbr;
+        const int32_t* rows_arg = plan_rows;
+        const uint32_t* mask_arg = plan_row_mask;
         int64_t no_arg = no, padded_arg = padded;
         int kvol_arg = kvol, begin_arg = sort_begin_bit;
         const int8_t* bitpos_arg = d_bitpos;
-        const unsigned* cnt_arg = scan_pending ? d_offset_cnt : nullptr;
+        const unsigned* cnt_arg = order_cnt;
         int32_t* tile_rows_arg = km->d.tile_rows;
         const int32_t* scan_cnt_arg = scan_pending ? cnt_a : nullptr;
         int64_t scan_m_arg = M;
@@ -1063,7 +1427,7 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
         int scan_nblk_arg = nblk;
         int64_t* scan_os_arg = d_offset_start;
         int64_t* scan_total_arg = d_totals + 1;
-        void* args[] = {&nbr_arg, &no_arg, &padded_arg, &kvol_arg, &bitpos_arg, &cnt_arg, &begin_arg, &rkeys, &rrows, &rkeys_sorted,
+        void* args[] = {&nbr_arg, &rows_arg, &mask_arg, &no_arg, &padded_arg, &kvol_arg, &bitpos_arg, &cnt_arg, &begin_arg, &rkeys, &rrows, &rkeys_sorted,
                         &rrows_b, &block_hist, &tile_rows_arg, &scan_cnt_arg, &scan_m_arg, &scan_excl_arg, &scan_nblk_arg, &scan_os_arg,
                         &scan_total_arg};
         // (with the scan on board the grid has one block more; the capacity test above leaves room for it)
@@ -1071,7 +1435,7 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
         SPCONV_CUDA_TRY(cudaLaunchCooperativeKernel(kernel, dim3(sort_blocks + (scan_pending ? 1 : 0)), dim3(kSortThreads), args, 0, stream));
       } else {
         if (scan_pending) k_scan_counts<<<1, 1024, 0, stream>>>(cnt_a, M, excl_a, nblk, kvol, d_offset_start, d_totals + 1, d_bitpos);
-        k_row_keys<<<rb, kBlock, 0, stream>>>(km->d.nbr, no, padded, kvol, d_bitpos, rkeys, rrows, km->d.tile_rows);
+        k_row_keys<<<rb, kBlock, 0, stream>>>(km->d.nbr, no, padded, kvol, d_bitpos, order_cnt, rkeys, rrows, km->d.tile_rows);
         SPCONV_CUDA_TRY(cub::DeviceRadixSort::SortPairs(cub_tmp, tmp_bytes, rkeys, rkeys_sorted, rrows, km->d.tile_rows, int(no),
                                                         sort_begin_bit, kvol, stream));
       }
@@ -1081,7 +1445,12 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     }
     SPCONV_STAGE(stages, "sort");
     if (after_sort) { const int e = after_sort(); if (e != SPCONV_OK) return e; }
-    if (kvol <= 32)
+    if (plan_rows != nullptr)
+      SPCONV_CUDA_TRY(launch_chained(k_tile_plan_rows, dim3(km->n_tiles), dim3(kTileRows), stream, static_cast<const int32_t*>(km->d.tile_rows),
+                                     plan_rows, kvol, km->d.tile_nbr, km->d.tile_crow, km->d.tile_mask, km->d.tile_absent, d_tile_blocks,
+                                     d_tiles_done, km->d.sorted_tiles, km->d.status, static_cast<const int64_t*>(d_totals),
+                                     int(totals_words), flag_target, counts_based ? 1 : 0));
+    else if (kvol <= 32)
       SPCONV_CUDA_TRY(launch_chained(k_tile_plan<true>, dim3(km->n_tiles), dim3(kTileRows), stream, km->d.tile_rows, km->d.nbr, no, kvol,
                                      km->mask_words, km->d.tile_nbr, km->d.tile_crow, km->d.tile_mask, km->d.tile_absent, d_tile_blocks,
                                      d_tiles_done, km->d.sorted_tiles, km->d.status, static_cast<const int64_t*>(d_totals),
@@ -1108,10 +1477,6 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   // ordinary synchronisation takes over.
   volatile int64_t* ready = h_totals + totals_words;
   const OffsetIndex offset_table = make_offset_index(K);
-  auto probe_line_enabled = [] {   // experiment switch (environment): SPCONV_KMAP_PROBE_LINE=0 uses k_subm_probe for every K
-    static const bool v = [] { const char* e = std::getenv("SPCONV_KMAP_PROBE_LINE"); return e == nullptr || std::atoi(e) != 0; }();
-    return v;
-  };
   auto expect_report = [&]() {
     *ready = 0;
     host.writer = stream;
@@ -1143,57 +1508,81 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   };
 
   SPCONV_CUDA_TRY(cudaMemsetAsync(d_totals, 0, (totals_words + 16) * sizeof(int64_t), stream));
-  SPCONV_CUDA_TRY(cudaMemsetAsync(keys1, 0xFF, size_t(cap1) * 8, stream));
+  SPCONV_CUDA_TRY(cudaMemsetAsync(table1, 0xFF, table_fill_bytes, stream));
 
-  if (submanifold) {
-    // Every size is known up front (n_out = n), so the whole map including the tile plan is enqueued before the
-    // host waits once, for the error word and the pair count; the pair lists, the only arrays whose size the
-    // host has to learn, are emitted after that wait and need no further one.
-    { const int e = allocate_map_arrays(n); if (e != SPCONV_OK) return e; }
+  if (known_outputs) {
+    // Every size is known up front (submanifold: n_out = n; inverse: the fine positions), so the whole map including
+    // the tile plan is enqueued before the host waits once, for the error word and the pair count.
+    { const int e = allocate_map_arrays(nq); if (e != SPCONV_OK) return e; }
     SPCONV_STAGE(stages, "alloc+memset");
-    SPCONV_CUDA_TRY(launch_chained(k_insert, dim3(nblk), dim3(kBlock), stream, coords4, int(n), keys1, vals1, cap1 - 1, d_status,
-                                   reinterpret_cast<int4*>(km->d.out_coords)));
+    SPCONV_HOST_TL("allocs+memsets");
+    int4* out_coords4 = reinterpret_cast<int4*>(km->d.out_coords);
+    if (n > 0)
+      SPCONV_CUDA_TRY(launch_chained(k_insert, dim3(nblk_in), dim3(kBlock), stream, coords4, int(n), table1, cap1 - 1, d_status,
+                                     (submanifold && !rows_table) ? out_coords4 : static_cast<int4*>(nullptr), occ));
     SPCONV_STAGE(stages, "insert");
-    if (K == 3 && probe_line_enabled())
-      SPCONV_CUDA_TRY(launch_chained(k_subm_probe_line<3>, dim3(nblk, 9), dim3(kBlock), stream, coords4, int(n), d, keys1, vals1, cap1 - 1,
-                                     km->d.nbr, cnt_a, d_offset_cnt, offset_table));
-    else
-      SPCONV_CUDA_TRY(launch_chained(k_subm_probe, grid_kn, dim3(kBlock), stream, coords4, int(n), K, d, keys1, vals1, cap1 - 1, km->d.nbr,
+    if (rows_table) {
+      // every offset of a row in one thread; also copies the rows' coordinates into the handle
+      auto probe_rows = [&](auto kernel) {
+        return launch_chained(kernel, dim3(nblk), dim3(kBlock), stream, qcoords4, int(nq), d, s, static_cast<const LocSlot*>(table1),
+                              cap1 - 1, static_cast<const uint32_t*>(occ), km->d.nbr, nbr_rows, row_mask,
+                              cnt_a, d_offset_cnt, out_coords4, d_status);
+      };
+      cudaError_t le = cudaErrorInvalidValue;
+      if (!inverse) le = K == 1 ? probe_rows(k_probe_rows<1, 0>) : probe_rows(k_probe_rows<3, 0>);
+      else le = K == 1 ? probe_rows(k_probe_rows<1, 1>) : K == 2 ? probe_rows(k_probe_rows<2, 1>) : probe_rows(k_probe_rows<3, 1>);
+      SPCONV_CUDA_TRY(le);
+      plan_rows = nbr_rows;
+      plan_row_mask = row_mask;
+    } else if (inverse) {
+      SPCONV_CUDA_TRY(cudaMemcpyAsync(km->d.out_coords, fine_coords, size_t(nq) * 16, cudaMemcpyDeviceToDevice, stream));
+      SPCONV_CUDA_TRY(launch_chained(k_inverse_probe, grid_kn, dim3(kBlock), stream, qcoords4, int(nq), K, s, d, static_cast<const LocSlot*>(table1),
+                                     cap1 - 1, km->d.nbr, cnt_a, d_offset_cnt, d_status, offset_table));
+    } else {
+      SPCONV_CUDA_TRY(launch_chained(k_subm_probe, grid_kn, dim3(kBlock), stream, coords4, int(n), K, d, static_cast<const LocSlot*>(table1), cap1 - 1, km->d.nbr,
                                      cnt_a, d_offset_cnt, offset_table));
+    }
     SPCONV_STAGE(stages, "probe");
-    // (the scan of the probe's pair counts rides along in the sort's launch)
-    // Pair lists: their exact size is only known on the device.  They are sized for 16 pairs per voxel (the
-    // workloads have 4-13) and their emission is enqueued behind the tile plan, before the host waits: it then
-    // runs while the host returns and launches whatever comes next.  A denser input gets exact lists and a
-    // second emission after the wait.
-    const int64_t pair_capacity = std::min<int64_t>(int64_t(kvol) * n, 16 * n);
+    SPCONV_HOST_TL("insert+probe");
+    // Pair lists: their exact size is only known on the device.  They are sized for 16 pairs per row (the
+    // workloads have 4-13); a denser input gets exact lists and a second emission after the wait.  Nothing on the
+    // way to the forward reads them, so their emission runs on a second stream beside the tile plan; the caller's
+    // stream joins that stream again behind whatever the caller's hook enqueues (the forward of spconv_layer), or
+    // at once.
+    const int64_t pair_capacity = std::min<int64_t>(int64_t(kvol) * nq, 16 * nq);
     { const int e = allocate_pairs(pair_capacity); if (e != SPCONV_OK) return e; }
-    // When the caller enqueues work behind the build's kernels (before_wait: the forward of spconv_layer), the
-    // emission, which that work does not need, leaves its way: it needs the offset table and the scan (both done
-    // when the sort's launch is), not the tile plan, so it runs on a second stream beside the tile plan, and the
-    // caller's stream joins it again only behind the caller's work.
     const bool hooked = before_wait != nullptr && *before_wait;
-    SideStream* side = hooked ? side_stream_for(km->device) : nullptr;
+    SideStream* side = side_stream_for(km->device);
     struct Rejoin {   // whatever happens after the fork, the caller's stream (which later frees the arrays) waits for the side stream
       cudaStream_t stream; SideStream* side; bool forked = false;
       ~Rejoin() { if (forked) { (void)cudaEventRecord(side->join, side->s); (void)cudaStreamWaitEvent(stream, side->join, 0); } }
     } rejoin{stream, side};
-    after_sort = [&]() -> int {
+    // The emission needs the offset table and the probe's hit counts, not the sort or the tile plan, so it is
+    // forked off behind the probe.  (Its blocks find their list positions themselves where per-offset totals
+    // exist; otherwise they need the scan of the per-block counts, which rides in the sort's launch, and the fork
+    // comes behind the sort.)
+    const int64_t* emit_excl = counts_based ? nullptr : excl_a;
+    auto fork_emit = [&]() -> int {
       if (side == nullptr) return SPCONV_OK;
       SPCONV_CUDA_TRY(cudaEventRecord(side->fork, stream));
       SPCONV_CUDA_TRY(cudaStreamWaitEvent(side->s, side->fork, 0));
       rejoin.forked = true;
-      k_subm_emit<<<grid_kn, kBlock, 0, side->s>>>(km->d.nbr, int(n), excl_a, km->d.pair_in, km->d.pair_out, pair_capacity);
+      k_subm_emit<<<grid_kn, kBlock, 0, side->s>>>(km->d.nbr, int(nq), emit_excl, cnt_a, d_offset_cnt, km->d.pair_in, km->d.pair_out, pair_capacity);
       SPCONV_CUDA_TRY(cudaEventRecord(side->join, side->s));
       return SPCONV_OK;
     };
+    if (counts_based) { const int e = fork_emit(); if (e != SPCONV_OK) return e; }
+    else after_sort = fork_emit;
+    SPCONV_HOST_TL("pairs+fork+emit");
     expect_report();
     flag_target = h_totals;
-    { const int e = enqueue_tile_plan(sa, cub_bytes, true); if (e != SPCONV_OK) return e; }
+    { const int e = enqueue_tile_plan(sa, cub_bytes, !counts_based); if (e != SPCONV_OK) return e; }
+    SPCONV_HOST_TL("sort+plan");
     flag_target = nullptr;
     after_sort = nullptr;
     if (side == nullptr)
-      SPCONV_CUDA_TRY(launch_chained(k_subm_emit, grid_kn, dim3(kBlock), stream, km->d.nbr, int(n), excl_a, km->d.pair_in, km->d.pair_out,
+      SPCONV_CUDA_TRY(launch_chained(k_subm_emit, grid_kn, dim3(kBlock), stream, static_cast<const int32_t*>(km->d.nbr), int(nq), emit_excl,
+                                     static_cast<const int32_t*>(cnt_a), static_cast<const unsigned*>(d_offset_cnt), km->d.pair_in, km->d.pair_out,
                                      pair_capacity));
     SPCONV_STAGE(stages, "schedule");
     if (hooked) { const int e = (*before_wait)(km); if (e != SPCONV_OK) return e; }
@@ -1201,14 +1590,17 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
       SPCONV_CUDA_TRY(cudaStreamWaitEvent(stream, side->join, 0));
       rejoin.forked = false;
     }
+    SPCONV_HOST_TL("before wait");
     { const int e = wait_for_report(); if (e != SPCONV_OK) return e; }
+    SPCONV_HOST_TL("after wait");
     SPCONV_STAGE(stages, "readback+sync");
     km->tile_blocks = h_totals[3];
     if (km->total_pairs > pair_capacity) {
       SPCONV_CUDA_TRY(cudaFreeAsync(km->d.pair_in, stream));
       km->d.pair_in = nullptr;
       { const int e = allocate_pairs(km->total_pairs); if (e != SPCONV_OK) return e; }
-      SPCONV_CUDA_TRY(launch_chained(k_subm_emit, grid_kn, dim3(kBlock), stream, km->d.nbr, int(n), excl_a, km->d.pair_in, km->d.pair_out,
+      SPCONV_CUDA_TRY(launch_chained(k_subm_emit, grid_kn, dim3(kBlock), stream, static_cast<const int32_t*>(km->d.nbr), int(nq), emit_excl,
+                                     static_cast<const int32_t*>(cnt_a), static_cast<const unsigned*>(d_offset_cnt), km->d.pair_in, km->d.pair_out,
                                      km->total_pairs));
     }
     SPCONV_STAGE(stages, "alloc+emit");
@@ -1219,8 +1611,8 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     const int pad = d * ((K - 1) / 2);
     SPCONV_CUDA_TRY(cudaMemsetAsync(keys2, 0xFF, size_t(cap2) * 8, stream));
     SPCONV_CUDA_TRY(cudaMemsetAsync(owner_cid, 0x7F, size_t(cap2) * 4, stream));
-    SPCONV_CUDA_TRY(launch_chained(k_insert, dim3(nblk), dim3(kBlock), stream, coords4, int(n), keys1, vals1, cap1 - 1, d_status,
-                                   static_cast<int4*>(nullptr)));
+    SPCONV_CUDA_TRY(launch_chained(k_insert, dim3(nblk), dim3(kBlock), stream, coords4, int(n), table1, cap1 - 1, d_status,
+                                   static_cast<int4*>(nullptr), static_cast<uint32_t*>(nullptr)));
     SPCONV_CUDA_TRY(launch_chained(k_strided_candidates, grid_kn, dim3(kBlock), stream, coords4, int(n), K, s, d, pad, keys2, owner_cid,
                                    cap2 - 1, cand_slot, cnt_a, d_status, offset_table));
     SPCONV_CUDA_TRY(launch_chained(k_scan_counts, dim3(1), dim3(1024), stream, static_cast<const int32_t*>(cnt_a), M, excl_a, nblk, kvol,
@@ -1240,15 +1632,20 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     SPCONV_CUDA_TRY(launch_chained(k_owner_assign, grid_kn, dim3(kBlock), stream, static_cast<const int32_t*>(cand_slot),
                                    static_cast<const int32_t*>(owner_cid), static_cast<const uint64_t*>(keys2), int(n),
                                    static_cast<const int64_t*>(excl_b), slot_out, reinterpret_cast<int4*>(km->d.out_coords)));
-    SPCONV_CUDA_TRY(launch_chained(k_strided_emit, grid_kn, dim3(kBlock), stream, static_cast<const int32_t*>(cand_slot),
-                                   static_cast<const int32_t*>(slot_out), int(n), km->n_out, static_cast<const int64_t*>(excl_a),
-                                   km->d.nbr, km->d.pair_in, km->d.pair_out));
     Scratch sort_scratch;
     sort_scratch.stream = stream;
     size_t cub2 = 0;
-    const size_t bytes = sort_bytes_for(no, &cub2) + 256;
+    const size_t bytes = sort_bytes_for(no, &cub2) + (rows_table ? pad256(size_t(no) * 128) : 0) + 512;
     SPCONV_CUDA_TRY(cudaMallocAsync(&sort_scratch.ptr, bytes, stream));
     Arena ta{static_cast<char*>(sort_scratch.ptr), bytes, 0};
+    if (rows_table) {
+      nbr_rows = ta.take<int32_t>(size_t(no) * 32);
+      SPCONV_CUDA_TRY(cudaMemsetAsync(nbr_rows, 0xFF, size_t(no) * 128, stream));
+      plan_rows = nbr_rows;
+    }
+    SPCONV_CUDA_TRY(launch_chained(k_strided_emit, grid_kn, dim3(kBlock), stream, static_cast<const int32_t*>(cand_slot),
+                                   static_cast<const int32_t*>(slot_out), int(n), km->n_out, static_cast<const int64_t*>(excl_a),
+                                   km->d.nbr, km->d.pair_in, km->d.pair_out, nbr_rows));
     expect_report();
     flag_target = h_totals;
     { const int e = enqueue_tile_plan(ta, cub2, false); if (e != SPCONV_OK) return e; }
@@ -1267,14 +1664,14 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
 // Offset table without any allocation (see spconv_subm_offset_table_noalloc in the header).
 //
 // The hash table lives in this fixed array, which every GPU that loads the library keeps until the
-// process exits.  Layout: keys [kNoAllocSlots] (8 bytes each) | values [kNoAllocSlots] (4 bytes each) |
-// one 256-byte block whose first word is the status word.
+// process exits.  Layout: kNoAllocSlots location-table slots of 16 bytes (key | row | unused) | one 256-byte block
+// whose first word is the status word.
 namespace spconv {
 namespace {
 
 constexpr uint32_t kNoAllocSlots = 2u * SPCONV_NOALLOC_MAX_VOXELS;   // power of two: at most half full
 static_assert((kNoAllocSlots & (kNoAllocSlots - 1)) == 0, "slot count must be a power of two");
-constexpr size_t kNoAllocBytes = size_t(kNoAllocSlots) * 8 + size_t(kNoAllocSlots) * 4 + 256;
+constexpr size_t kNoAllocBytes = size_t(kNoAllocSlots) * sizeof(LocSlot) + 256;
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
@@ -1284,8 +1681,8 @@ std::mutex g_noalloc_mu;
 unsigned char* g_noalloc_ptr[64] = {nullptr};
 
 // Same probing as k_subm_probe, without the per-block hit counts (they would need more scratch).
-__global__ void k_subm_probe_only(const int4* __restrict__ coords, int n, int K, int dil, const uint64_t* __restrict__ keys,
-                                  const int32_t* __restrict__ vals, uint32_t capmask, int32_t* __restrict__ nbr,
+__global__ void k_subm_probe_only(const int4* __restrict__ coords, int n, int K, int dil, const LocSlot* __restrict__ table,
+                                  uint32_t capmask, int32_t* __restrict__ nbr,
                                   const __grid_constant__ OffsetIndex index) {
   const int k = blockIdx.y;
   const int j = blockIdx.x * kBlock + threadIdx.x;
@@ -1298,7 +1695,7 @@ __global__ void k_subm_probe_only(const int4* __restrict__ coords, int n, int K,
   const int x = c.y + dx, y = c.z + dy, z = c.w + dz;
   int v = -1;
   if ((dx | dy | dz) == 0) v = j;
-  else if (in_range(x) && in_range(y) && in_range(z)) v = table_find(keys, vals, capmask, pack_key(c.x, x, y, z));
+  else if (in_range(x) && in_range(y) && in_range(z)) v = table_find(table, capmask, pack_key(c.x, x, y, z));
   nbr[size_t(k) * n + j] = v;
 }
 
@@ -1329,19 +1726,18 @@ extern "C" int spconv_subm_offset_table_noalloc(const int32_t* coords, int64_t n
     }
     base = g_noalloc_ptr[dev];
   }
-  uint64_t* keys = reinterpret_cast<uint64_t*>(base);
-  int32_t* vals = reinterpret_cast<int32_t*>(base + size_t(kNoAllocSlots) * 8);
-  uint32_t* status = reinterpret_cast<uint32_t*>(base + size_t(kNoAllocSlots) * 12);
+  LocSlot* table = reinterpret_cast<LocSlot*>(base);
+  uint32_t* status = reinterpret_cast<uint32_t*>(base + size_t(kNoAllocSlots) * sizeof(LocSlot));
 
   // The array keeps whatever the previous call left: empty the slots this call will probe and the status word.
   const int K = kernel_size, kvol = K * K * K;
   const uint32_t cap = pow2_at_least(uint64_t(2) * n);
   const int nblk = int((n + kBlock - 1) / kBlock);
-  SPCONV_CUDA_TRY(cudaMemsetAsync(keys, 0xFF, size_t(cap) * 8, stream));
+  SPCONV_CUDA_TRY(cudaMemsetAsync(table, 0xFF, size_t(cap) * sizeof(LocSlot), stream));
   SPCONV_CUDA_TRY(cudaMemsetAsync(status, 0, 256, stream));
   const int4* coords4 = reinterpret_cast<const int4*>(coords);
-  k_insert<<<nblk, kBlock, 0, stream>>>(coords4, int(n), keys, vals, cap - 1, status, nullptr);
-  k_subm_probe_only<<<dim3(nblk, kvol), kBlock, 0, stream>>>(coords4, int(n), K, dilation, keys, vals, cap - 1, nbr_out, make_offset_index(K));
+  k_insert<<<nblk, kBlock, 0, stream>>>(coords4, int(n), table, cap - 1, status, nullptr);
+  k_subm_probe_only<<<dim3(nblk, kvol), kBlock, 0, stream>>>(coords4, int(n), K, dilation, table, cap - 1, nbr_out, make_offset_index(K));
   SPCONV_CUDA_TRY(cudaGetLastError());
   uint32_t st = 0;
   SPCONV_CUDA_TRY(cudaMemcpyAsync(&st, status, sizeof(st), cudaMemcpyDeviceToHost, stream));

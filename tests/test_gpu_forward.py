@@ -244,12 +244,14 @@ print("ok")
 
 @pytest.mark.gpu
 def test_tile_plan_sort_paths_agree():
-    """The cooperative key-and-sort launch and the library radix sort are both stable sorts of the same keys, so
-    they must cut the rows into identical tiles (the switch is read once per process, hence the child process);
-    either plan must hold every output row exactly once and give the oracle's result."""
+    """The two ways the tile plan sorts the rows -- grid-wide in one cooperative launch, and the library's radix sort
+    (the switch is read once per process, hence the child processes) -- are stable sorts of the same keys, so they
+    must cut the rows into identical tiles; every plan must hold every output row exactly once, pack a LiDAR sweep
+    into few (tile, offset) blocks, and give the oracle's result."""
     import os
     import subprocess
     import sys
+    import tempfile
     code = f"""
 import sys, numpy as np, torch
 sys.path.insert(0, {os.path.dirname(os.path.dirname(os.path.abspath(__file__)))!r}); sys.path.insert(0, {os.path.dirname(os.path.abspath(__file__))!r})
@@ -261,24 +263,27 @@ km, _ = check_layer(coords, lay, algo="tcgen05")
 rows = km.tile_rows.cpu().numpy().ravel()
 live = np.sort(rows[rows >= 0])
 assert np.array_equal(live, np.arange(km.n_out)), "every output row exactly once"
-assert (rows < 0).sum() == rows.size - km.n_out, "only the padding of the last tile is negative"
-np.save(sys.argv[1], km.tile_rows.cpu().numpy())
+assert (rows < 0).sum() == rows.size - km.n_out and (rows[km.n_out:] < 0).all(), "only the padding of the last tile is negative"
 lay["kind"], lay["stride"] = "spconv", 2
-check_layer(coords, lay, algo="tcgen05")
+km2, _ = check_layer(coords, lay, algo="tcgen05")
+sweep = wl.lidar_sweep(3)
+km3, _ = check_layer(sweep, dict(kind="subm", kernel=3, stride=1, dilation=1, cin=64, cout=64, dtype="bf16"), algo="tcgen05", sample_rows=2000)
+assert km3.tile_blocks < 12 * km3.n_tiles, (km3.tile_blocks, km3.n_tiles)    # input order: about 25 blocks per tile
+np.savez(sys.argv[1], a=km.tile_rows.cpu().numpy(), b=km2.tile_rows.cpu().numpy(), c=km3.tile_rows.cpu().numpy())
 print("ok")
 """
-    import tempfile
-    import numpy as np
     plans = []
-    for library_sort in ("0", "1"):
-        with tempfile.NamedTemporaryFile(suffix=".npy", delete=False) as f:
+    for env in ({}, {"SPCONV_KMAP_LIBRARY_SORT": "1"}):
+        with tempfile.NamedTemporaryFile(suffix=".npz", delete=False) as f:
             path = f.name
-        env = dict(os.environ, SPCONV_KMAP_LIBRARY_SORT=library_sort)
-        res = subprocess.run([sys.executable, "-c", code, path], env=env, capture_output=True, text=True, timeout=300)
-        assert res.returncode == 0 and "ok" in res.stdout, res.stdout[-2000:] + res.stderr[-2000:]
-        plans.append(np.load(path))
+        res = subprocess.run([sys.executable, "-c", code, path], env=dict(os.environ, **env), capture_output=True, text=True, timeout=600)
+        assert res.returncode == 0 and "ok" in res.stdout, str(env) + res.stdout[-2000:] + res.stderr[-2000:]
+        with np.load(path) as z:
+            plans.append({k: z[k] for k in z.files})
         os.unlink(path)
-    assert np.array_equal(plans[0], plans[1])
+    for other in plans[1:]:
+        for k in plans[0]:
+            assert np.array_equal(plans[0][k], other[k]), k
 
 
 @pytest.mark.gpu
