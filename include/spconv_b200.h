@@ -257,6 +257,33 @@ int spconv_layer_host(const int32_t* coords_host, int64_t n, const void* feats_h
 int spconv_subm_offset_table_noalloc(const int32_t* coords, int64_t n, int kernel_size, int dilation,
                                      int32_t* nbr_out, void* cuda_stream);
 
+/*
+ * Diagnostics: copy the 16 status words that device kernels of this kernel map write to host memory `out16`
+ * (synchronous copy).  Word 0: status bits (8 = a bounded wait of the tensor-core forward ran out); word 1: code of
+ * the first wait that gave up (role << 24 | step, top bit set); word 2: its CTA + 1.  Cleared by the next build of a
+ * tile plan and, word 0 only, by spconv_last_device_status.
+ */
+int spconv_kmap_status_words(const spconv_kmap_t* kmap, uint32_t* out16 /* host */);
+
+/*
+ * Test hooks.  Not for production use: they exist so that tests can reach the failure paths that no valid input
+ * reaches, without faulting or hanging the device.  Process-wide, take effect for calls made afterwards; value 0
+ * restores the normal behaviour.
+ *   SPCONV_HOOK_TABLE_SLOTS         force the location table to pow2(value) slots, whatever the input: with fewer
+ *                                   slots than rows the bounded probe sequence runs out and the build returns
+ *                                   SPCONV_ERR_TABLE_FULL.
+ *   SPCONV_HOOK_PIPE_WAIT_LIMIT_US  shorten the time bound of every wait inside the tensor-core forward to `value`
+ *                                   microseconds and withhold the weights of the first step of CTA 0, so that one
+ *                                   wait runs out: the kernel gives up by itself and the status word reports
+ *                                   SPCONV_ERR_PIPE_TIMEOUT.
+ * Two more switches are environment variables read once per process: SPCONV_TC_MAX_CTAS=<n> caps the grid of the
+ * tensor-core forward (small inputs then exercise many tiles per CTA and several rounds), and
+ * SPCONV_KMAP_LIBRARY_SORT=1 sorts the tile plan's rows with the CUDA library's radix sort instead of the fused
+ * cooperative launch (the path very large maps take).
+ */
+typedef enum { SPCONV_HOOK_TABLE_SLOTS = 1, SPCONV_HOOK_PIPE_WAIT_LIMIT_US = 2 } spconv_test_hook_t;
+int spconv_test_hook(int which, long long value);
+
 /* Static, never-NULL description of a status code. */
 const char* spconv_strerror(int status);
 

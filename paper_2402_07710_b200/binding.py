@@ -23,7 +23,9 @@ DTYPE_BY_NAME = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloa
 EXPORTS = (
     "spconv_build_kmap", "spconv_build_inverse_kmap", "spconv_kmap_info", "spconv_kmap_destroy", "spconv_forward", "spconv_forward_algo",
     "spconv_last_device_status", "spconv_layer", "spconv_layer_host", "spconv_strerror", "spconv_subm_offset_table_noalloc",
+    "spconv_kmap_status_words", "spconv_test_hook",
 )
+HOOK_TABLE_SLOTS, HOOK_PIPE_WAIT_LIMIT_US = 1, 2
 NOALLOC_MAX_VOXELS = 131072
 
 
@@ -80,6 +82,10 @@ def load() -> ctypes.CDLL:
                                           ctypes.POINTER(i64), vp]
         lib.spconv_subm_offset_table_noalloc.restype = i32
         lib.spconv_subm_offset_table_noalloc.argtypes = [vp, i64, i32, i32, vp, vp]
+        lib.spconv_kmap_status_words.restype = i32
+        lib.spconv_kmap_status_words.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+        lib.spconv_test_hook.restype = i32
+        lib.spconv_test_hook.argtypes = [i32, ctypes.c_longlong]
         lib.spconv_strerror.restype = ctypes.c_char_p
         lib.spconv_strerror.argtypes = [i32]
         _lib = lib
@@ -263,6 +269,22 @@ def spconv_layer(coords: torch.Tensor, feats: torch.Tensor, weights: torch.Tenso
 
 def spconv_last_device_status(kmap: Kmap, stream=None) -> int:
     return int(load().spconv_last_device_status(kmap._h, ctypes.c_void_p(_stream_ptr(stream))))
+
+
+def spconv_kmap_status_words(kmap: Kmap) -> list:
+    """The 16 status words device kernels of this map wrote (diagnostics)."""
+    words = (ctypes.c_uint32 * 16)()
+    st = load().spconv_kmap_status_words(kmap._h, words)
+    if st != 0:
+        raise SpconvError(st, "spconv_kmap_status_words")
+    return list(words)
+
+
+def spconv_test_hook(which: int, value: int) -> None:
+    """Test hooks of the library (see the header); value 0 restores normal behaviour."""
+    st = load().spconv_test_hook(int(which), int(value))
+    if st != 0:
+        raise SpconvError(st, "spconv_test_hook")
 
 
 def spconv_layer_host(coords: torch.Tensor, feats: torch.Tensor, weights: torch.Tensor, stride: int, dilation: int,

@@ -240,14 +240,23 @@ int spconv_layer_host(const int32_t* coords_host, int64_t n, const void* feats_h
   return spconv_last_device_status(km, stream);
 }
 
-// Not part of the public header: copies the 16 status words of a kernel map to host memory (word 0 status bits,
-// word 1 code of the first wait that gave up, word 2 its CTA + 1).
-int spconv_internal_read_status(const spconv_kmap_t* km, uint32_t* out16) {
-  if (km == nullptr || km->d.status == nullptr) return SPCONV_ERR_INVALID_ARG;
+int spconv_kmap_status_words(const spconv_kmap_t* km, uint32_t* out16) {
+  if (km == nullptr || out16 == nullptr) return SPCONV_ERR_INVALID_ARG;
+  if (km->d.status == nullptr) { std::memset(out16, 0, 64); return SPCONV_OK; }
   return cudaMemcpy(out16, km->d.status, 64, cudaMemcpyDeviceToHost) == cudaSuccess ? SPCONV_OK : SPCONV_ERR_CUDA;
 }
 
-// Not part of the public header: profiling hook used by development scripts (see forward_tc.cu).
+int spconv_test_hook(int which, long long value) {
+  switch (which) {
+    case SPCONV_HOOK_TABLE_SLOTS: set_kmap_test_table_slots(value); return SPCONV_OK;
+    case SPCONV_HOOK_PIPE_WAIT_LIMIT_US: set_forward_tc_test_wait_limit_us(value); return SPCONV_OK;
+  }
+  return SPCONV_ERR_INVALID_ARG;
+}
+
+#ifdef SPCONV_TC_PROFILE
+// Development builds only: per-CTA timeline buffer of the tensor-core forward (see forward_tc.cu).
 void spconv_internal_set_timeline(void* device_buffer) { set_forward_tc_timeline(static_cast<unsigned long long*>(device_buffer)); }
+#endif
 
 }  // extern "C"

@@ -63,6 +63,7 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
                     cudaStream_t stream, spconv_kmap** out, const std::function<int(spconv_kmap*)>* before_wait = nullptr,
                     const int32_t* fine_coords = nullptr, int64_t n_fine = 0);
 void destroy_kmap_impl(spconv_kmap* km);
+void set_kmap_test_table_slots(long long slots);          // test hook, see spconv_test_hook
 
 // forward_simt.cu
 int forward_simt(const void* feats, const void* w, const spconv_kmap* km, void* out, int cin, int cout,
@@ -71,6 +72,7 @@ int forward_simt(const void* feats, const void* w, const spconv_kmap* km, void* 
 // forward_tc.cu
 bool forward_tc_supported(int cin, int cout, spconv_dtype_t dtype);
 void set_forward_tc_timeline(unsigned long long* buf);
+void set_forward_tc_test_wait_limit_us(long long us);     // test hook, see spconv_test_hook
 // strict_order: the kernel map may still be under construction by work that precedes the launch in the stream
 // (the launch comes from build_kmap_impl's before_wait), so the kernel must not read it ahead of that work.
 int forward_tc(const void* feats, const void* w, const spconv_kmap* km, void* out, int cin, int cout,

@@ -8,6 +8,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace spconv {
@@ -99,11 +101,86 @@ k_forward_simt(const T* __restrict__ feats, const T* __restrict__ w, const int32
   }
 }
 
+
+// fp32 fast path: all weights in shared memory, four output channels per thread, rows straight from global memory.
+// The weights of every offset are staged once per block as they lie in memory ([K^3][Cin][Cout]); cout / 4
+// neighbouring threads share an output row and each keeps four of its channels in registers; a thread fetches the
+// row's offset-table entries 32 at a time (one round trip), then walks the offsets in ascending order and, where
+// the row has an input, reads that input row with 16-byte loads (the threads of a row read the same addresses: one
+// request) and multiplies it with 16-byte reads of the offset's weights.  Rows are independent, so apart from the
+// one barrier behind the staging nothing waits for anything but its own loads; the result leaves as one 16-byte
+// store per thread.  Taken when the weights fit (kvol * cin * cout * 4 bytes within the SM's shared memory).
+constexpr int kRowsThreads = 256;
+__global__ void __launch_bounds__(kRowsThreads)
+k_forward_rows_f32(const float* __restrict__ feats, const float* __restrict__ w, const int32_t* __restrict__ nbr, int64_t n_out,
+                   int kvol, int cin, int cout, float* __restrict__ out) {
+  extern __shared__ __align__(16) float wsm[];   // [kvol][cin][cout]
+  const int tid = threadIdx.x;
+  const int tpr = cout >> 2;                       // threads per row
+  const int rows_per_block = kRowsThreads / tpr;
+  const int r = tid / tpr, t = tid - r * tpr;
+  const int64_t row = int64_t(blockIdx.x) * rows_per_block + r;
+  const bool live = r < rows_per_block && row < n_out;
+  {
+    const float4* src = reinterpret_cast<const float4*>(w);
+    float4* dst = reinterpret_cast<float4*>(wsm);
+    const int total4 = (kvol * cin * cout) >> 2;
+    for (int i = tid; i < total4; i += kRowsThreads) dst[i] = __ldg(src + i);
+  }
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  const int cin4 = cin >> 2;
+  for (int k0 = 0; k0 < kvol; k0 += 32) {
+    int idx[32];
+#pragma unroll
+    for (int u = 0; u < 32; ++u) idx[u] = (live && k0 + u < kvol) ? __ldg(nbr + size_t(k0 + u) * n_out + row) : -1;
+    if (k0 == 0) __syncthreads();   // the weights are staged (the first entries were requested before the wait)
+#pragma unroll
+    for (int u = 0; u < 32; ++u) {
+      if (idx[u] < 0) continue;
+      const float4* xr = reinterpret_cast<const float4*>(feats + size_t(idx[u]) * cin);
+      const float* wk = wsm + size_t(k0 + u) * cin * cout + 4 * t;
+      for (int c4 = 0; c4 < cin4; ++c4) {
+        const float4 xv = __ldg(xr + c4);
+        const float4 w0 = *reinterpret_cast<const float4*>(wk + size_t(4 * c4 + 0) * cout);
+        const float4 w1 = *reinterpret_cast<const float4*>(wk + size_t(4 * c4 + 1) * cout);
+        const float4 w2 = *reinterpret_cast<const float4*>(wk + size_t(4 * c4 + 2) * cout);
+        const float4 w3 = *reinterpret_cast<const float4*>(wk + size_t(4 * c4 + 3) * cout);
+        acc.x = fmaf(xv.x, w0.x, acc.x); acc.y = fmaf(xv.x, w0.y, acc.y); acc.z = fmaf(xv.x, w0.z, acc.z); acc.w = fmaf(xv.x, w0.w, acc.w);
+        acc.x = fmaf(xv.y, w1.x, acc.x); acc.y = fmaf(xv.y, w1.y, acc.y); acc.z = fmaf(xv.y, w1.z, acc.z); acc.w = fmaf(xv.y, w1.w, acc.w);
+        acc.x = fmaf(xv.z, w2.x, acc.x); acc.y = fmaf(xv.z, w2.y, acc.y); acc.z = fmaf(xv.z, w2.z, acc.z); acc.w = fmaf(xv.z, w2.w, acc.w);
+        acc.x = fmaf(xv.w, w3.x, acc.x); acc.y = fmaf(xv.w, w3.y, acc.y); acc.z = fmaf(xv.w, w3.z, acc.z); acc.w = fmaf(xv.w, w3.w, acc.w);
+      }
+    }
+  }
+  if (live) *reinterpret_cast<float4*>(out + size_t(row) * cout + 4 * t) = acc;
+}
+
 }  // namespace
 
 int forward_simt(const void* feats, const void* w, const spconv_kmap* km, void* out, int cin, int cout,
                  spconv_dtype_t dtype, cudaStream_t stream) {
   if (km->n_out == 0) return SPCONV_OK;
+  // fp32 with weights that fit shared memory: the all-weights-resident kernel
+  const size_t w_bytes = size_t(km->kvol) * cin * cout * 4;
+  if (dtype == SPCONV_F32 && cin % 4 == 0 && cout % 4 == 0 && cout >= 4 && cout <= 4 * kRowsThreads && w_bytes <= size_t(200) * 1024) {
+    static std::mutex mu;
+    static size_t smem_set[64] = {0};   // largest dynamic shared memory size enabled so far, per device
+    const int dev = km->device;
+    if (dev < 0 || dev >= 64) return SPCONV_ERR_INVALID_ARG;
+    if (w_bytes > 48 * 1024) {
+      std::lock_guard<std::mutex> lock(mu);
+      if (smem_set[dev] < w_bytes) {
+        SPCONV_CUDA_TRY(cudaFuncSetAttribute(k_forward_rows_f32, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        smem_set[dev] = size_t(200) * 1024;
+      }
+    }
+    const int rows_per_block = kRowsThreads / (cout / 4);
+    const unsigned row_blocks = unsigned((km->n_out + rows_per_block - 1) / rows_per_block);
+    k_forward_rows_f32<<<row_blocks, kRowsThreads, w_bytes, stream>>>(static_cast<const float*>(feats), static_cast<const float*>(w), km->d.nbr,
+                                                                      km->n_out, km->kvol, cin, cout, static_cast<float*>(out));
+    SPCONV_CUDA_TRY(cudaGetLastError());
+    return SPCONV_OK;
+  }
   const unsigned blocks = unsigned((km->n_out + kRows - 1) / kRows);
   switch (dtype) {
     case SPCONV_F32:

@@ -33,6 +33,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -76,7 +77,7 @@ constexpr bool grouped_shape(int cin, int cout) { return kGroupSteps && cin <= k
 constexpr int kMaxAStages = SPCONV_TC_ASTAGES;
 constexpr int kMaxGroup = 32;                    // tiles a CTA keeps in TMEM at once (<= 512 / COUT)
 constexpr uint32_t kSpinLimit = 1u << 24;        // polls per wait, and
-constexpr uint64_t kWaitLimitNs = 250ull * 1000 * 1000;  // wall-time bound per wait (0.25 s)
+constexpr uint64_t kWaitLimitNs = 250ull * 1000 * 1000;  // wall-time bound per wait (0.25 s) unless a test shortens it
 constexpr int kMaxSmem = 227 * 1024;             // largest dynamic shared memory a CTA may request on sm_100
 constexpr int kStagingPitch = 64 * 2 + 16;       // epilogue staging row: 64 columns of 16 bits + one 16-byte pad
 
@@ -213,29 +214,35 @@ __device__ __forceinline__ void mbar_test_wait3(uint32_t bar0, uint32_t par0, ui
       : "r"(bar0), "r"(par0), "r"(bar1), "r"(par1), "r"(bar2), "r"(par2)
       : "memory");
 }
-// Bounded wait: at most kSpinLimit polls and at most kWaitLimitNs of wall time.  Returns false when a
+// What every bounded wait of a CTA needs: the CTA's give-up flag, the kernel map's status words, the time limit.
+struct WaitCtx {
+  volatile int* abort_flag;
+  uint32_t* diag;
+  uint64_t limit_ns;
+};
+// Bounded wait: at most kSpinLimit polls and at most limit_ns of wall time.  Returns false when a
 // bound was hit or another thread of the CTA already gave up.
 // `where` identifies the wait (role << 24 | detail); the first wait of the CTA that gives up records it in
 // the kernel map's status words 1 (code) and 2 (CTA + 1), first writer wins, for post-mortem reading.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* diag, uint32_t where) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& ctx, uint32_t where) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer_ns();
   for (uint32_t it = 0; it < kSpinLimit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if ((it & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) break;
+    if (*ctx.abort_flag) return false;
+    if ((it & 63u) == 63u && global_timer_ns() - t0 > ctx.limit_ns) break;
   }
-  if (atomicExch(const_cast<int*>(abort_flag), 1) == 0) {
-    atomicCAS(diag + 1, 0u, where | 0x80000000u);
-    atomicCAS(diag + 2, 0u, blockIdx.x + 1u);
+  if (atomicExch(const_cast<int*>(ctx.abort_flag), 1) == 0) {
+    atomicCAS(ctx.diag + 1, 0u, where | 0x80000000u);
+    atomicCAS(ctx.diag + 2, 0u, blockIdx.x + 1u);
   }
   return false;
 }
 // Warp-wide bounded wait: lane 0 polls, the other lanes take its verdict (they are ordered behind lane 0's
 // acquire by the warp-level synchronisation of the shuffle).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t* diag, uint32_t where) {
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, const WaitCtx& ctx, uint32_t where) {
   bool ok = true;
-  if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, diag, where);
+  if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, ctx, where);
   return __shfl_sync(0xffffffffu, int(ok), 0) != 0;
 }
 __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
@@ -340,7 +347,8 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
              const uint32_t* __restrict__ tile_mask, const uint32_t* __restrict__ tile_absent,
              const int32_t* __restrict__ sorted_tiles, uint8_t* __restrict__ out,
              int n_tiles, int kvol, int mask_words, int G, int n_rounds, uint32_t tmem_cols, uint32_t idesc, int is_bf16,
-             uint32_t* __restrict__ status, unsigned long long* __restrict__ timeline, long long feat_lines, int strict_order) {
+             uint32_t* __restrict__ status, unsigned long long* __restrict__ timeline, long long feat_lines, int strict_order,
+             unsigned long long wait_limit_ns, int withhold_first_w) {
   using C = Cfg<CIN, COUT, GROUPED>;
   extern __shared__ uint8_t smem_raw[];
   // Swizzled operand tiles need 1024-byte aligned bases.
@@ -354,6 +362,7 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abort_flag = &sm->abort_flag;
+  const WaitCtx wctx{abort_flag, status, wait_limit_ns};
   // Optional per-CTA timeline (diagnostics): globaltimer stamps when a buffer is installed.
   auto stamp = [&](int slot) { if (timeline != nullptr) timeline[size_t(blockIdx.x) * 16 + slot] = global_timer_ns(); };
   if (tid == 0) stamp(0);
@@ -592,7 +601,7 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
 
     // =============================== epilogue (every warp that has staging room, once its role is done) ===============================
     auto run_epilogue = [&](bool ok) {
-      if (ok) { ok = mbar_wait_warp(smem_u32(&sm->accum_full), accum_uses & 1u, abort_flag, status, 2u << 24); ++accum_uses; }
+      if (ok) { ok = mbar_wait_warp(smem_u32(&sm->accum_full), accum_uses & 1u, wctx, 2u << 24); ++accum_uses; }
       tc_fence_after();
       if (tid == 0 && round == 0) stamp(4);
       if (ok) {
@@ -747,7 +756,7 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
           SPCONV_PROF_T(c0);
           // every lane polls (one warp instruction, no divergence); measured faster than one lane plus a broadcast
           if (!__all_sync(0xffffffffu, mbar_test_wait(smem_u32(&sm->empty_a[stage]), parity))) {
-            ok = mbar_wait_warp(smem_u32(&sm->empty_a[stage]), parity, abort_flag, status, (1u << 24) | uint32_t(m));
+            ok = mbar_wait_warp(smem_u32(&sm->empty_a[stage]), parity, wctx, (1u << 24) | uint32_t(m));
             if (!ok) continue;
           }
           SPCONV_PROF_T(c1);
@@ -848,7 +857,7 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
             const uint32_t g = word & 31u;
             const int n_sub = int((word >> 5) & 7u) + 1;
             SPCONV_PROF_T(m0);
-            ok = mbar_wait(full_a0 + mma_stage * 8u, mma_phase, abort_flag, status, (4u << 24) | uint32_t(m));
+            ok = mbar_wait(full_a0 + mma_stage * 8u, mma_phase, wctx, (4u << 24) | uint32_t(m));
             if (!ok) break;
             SPCONV_PROF_T(m1);
             fence_proxy_async();
@@ -886,7 +895,7 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
             const bool group_ends = m + 1 == n_walk || ((e_next >> 5) & 127u) != ((e >> 5) & 127u);
             const bool mine = (e >> kStepIssuerShift) == me;
             if ((mine || group_ends) && !w_known) {
-              ok = mbar_wait(full_w0 + mma_wslot * 8u, mma_wphase, abort_flag, status, (3u << 24) | uint32_t(m));
+              ok = mbar_wait(full_w0 + mma_wslot * 8u, mma_wphase, wctx, (3u << 24) | uint32_t(m));
               if (!ok) break;
               w_known = true;
             }
@@ -902,10 +911,10 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
           const bool w_done = C::kWInStage ? false : C::kSharedW ? (m + 1 == n_walk || ((e_next >> 5) & 127u) != ((e >> 5) & 127u)) : (e & kStepLast) != 0u;
           SPCONV_PROF_T(m0);
           if (!C::kSharedW && !C::kWInStage && (e & kStepFirst)) {
-            ok = mbar_wait(full_w0 + mma_wslot * 8u, mma_wphase, abort_flag, status, (3u << 24) | uint32_t(m));
+            ok = mbar_wait(full_w0 + mma_wslot * 8u, mma_wphase, wctx, (3u << 24) | uint32_t(m));
             if (!ok) break;
           }
-          ok = mbar_wait(full_a0 + mma_stage * 8u, mma_phase, abort_flag, status, (4u << 24) | uint32_t(m));
+          ok = mbar_wait(full_a0 + mma_stage * 8u, mma_phase, wctx, (4u << 24) | uint32_t(m));
           if (!ok) break;
           SPCONV_PROF_T(m1);
           fence_proxy_async();   // the rows were written by cp.async; the MMA reads them through the async proxy
@@ -964,10 +973,11 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
             const uint32_t word = gsteps[m];
             const int n_sub = int((word >> 5) & 7u) + 1;
             const uint32_t wslot = me * uint32_t(C::kStagesPer) + w_group % uint32_t(C::kStagesPer), wuse = w_group / uint32_t(C::kStagesPer);
-            ok = mbar_wait(smem_u32(&sm->empty_a[wslot]), (wuse & 1u) ^ 1u, abort_flag, status, (5u << 24) | uint32_t(m));
+            ok = mbar_wait(smem_u32(&sm->empty_a[wslot]), (wuse & 1u) ^ 1u, wctx, (5u << 24) | uint32_t(m));
             if (!ok) break;
             const uint32_t bar = smem_u32(&sm->full_a[wslot]);
             const uint32_t dst = smem_u32(w_ring + wslot * C::kWSlotBytes);
+            if (withhold_first_w && blockIdx.x == 0 && me == 0 && m == 0 && round == 0) { ++w_group; continue; }   // test hook, see launch()
             mbar_arrive_expect_tx(bar, uint32_t(n_sub * C::kWBytesRaw));
             for (int sidx = 0; sidx < n_sub; ++sidx) {
               const int k = int((word >> (8 + 6 * sidx)) & 63u);
@@ -987,12 +997,13 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
           // kWInStage: W_k goes into the stage of the step itself, behind the same two barriers as its rows
           const uint32_t depth = uint32_t(C::kWInStage ? C::kStagesPer : C::kWStagesPer);
           const uint32_t wslot = (C::kSharedW ? 0u : me * depth) + w_group % depth, wuse = w_group / depth;
-          ok = mbar_wait(smem_u32(C::kWInStage ? &sm->empty_a[wslot] : &sm->empty_w[wslot]), (wuse & 1u) ^ 1u, abort_flag, status, (5u << 24) | uint32_t(m));
+          ok = mbar_wait(smem_u32(C::kWInStage ? &sm->empty_a[wslot] : &sm->empty_w[wslot]), (wuse & 1u) ^ 1u, wctx, (5u << 24) | uint32_t(m));
           if (!ok) break;
           SPCONV_PROF_T(w1);
           SPCONV_PROF_ADD(wc_wait, w0, w1);
           const uint32_t bar = smem_u32(C::kWInStage ? &sm->full_a[wslot] : &sm->full_w[wslot]);
           const uint32_t dst = smem_u32(w_ring + wslot * C::kWSlotBytes);
+          if (withhold_first_w && blockIdx.x == 0 && me == 0 && m == 0 && round == 0) { ++w_group; continue; }   // test hook, see launch()
           mbar_arrive_expect_tx(bar, uint32_t(C::kWBytesRaw));
 #pragma unroll
           for (int p = 0; p < C::kWPanels; ++p) tma_load_2d(dst + p * C::kWPanelBytes, &w_map, bar, p * 64, k * CIN);
@@ -1025,7 +1036,7 @@ k_forward_tc(const __grid_constant__ CUtensorMap w_map, const uint8_t* __restric
     const uint64_t t0 = global_timer_ns();
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
       if (mbar_try_wait(smem_u32(&sm->drain), 0u)) break;
-      if ((it & 63u) == 63u && global_timer_ns() - t0 > kWaitLimitNs) break;
+      if ((it & 63u) == 63u && global_timer_ns() - t0 > wait_limit_ns) break;
     }
   }
   if (warp < C::kProducerWarps) cp_async_wait_all();
@@ -1069,14 +1080,13 @@ int max_ctas_override() {
   return v;
 }
 
-// Experiment switch (environment): SPCONV_TC_PREFETCH_ROWS=0 turns the up-front L2 request for the input rows off.
-bool prefetch_rows_enabled() {
-  static const bool v = [] {
-    const char* e = std::getenv("SPCONV_TC_PREFETCH_ROWS");
-    return e == nullptr || std::atoi(e) != 0;
-  }();
-  return v;
-}
+// Test hook for the kernel's give-up path (spconv_test_hook, SPCONV_HOOK_PIPE_WAIT_LIMIT_US): a positive value
+// shortens the wall-time bound of every wait to that many microseconds and makes CTA 0's first W loader withhold the
+// weights of its first step, so that the wait for that step's stage runs out, the CTA gives up, frees what it holds
+// and the launch reports SPCONV_ERR_PIPE_TIMEOUT through the status word -- nothing faults and nothing waits without
+// a bound.  0: the ordinary limit, nothing withheld.
+std::atomic<long long> g_test_wait_limit_us{0};
+long long test_wait_limit_us() { return g_test_wait_limit_us.load(std::memory_order_relaxed); }
 
 template <int CIN, int COUT, bool GROUPED>
 size_t smem_bytes_for(int kvol) {
@@ -1147,12 +1157,17 @@ int launch(const void* feats, const void* w, const spconv_kmap* km, void* out, s
 
   // Input rows the kernel requests into L2 up front, in 128-byte lines: all of them up to 32 MB.
   const long long feat_bytes = (long long)km->n_in * C::kARowBytes;
-  const long long feat_lines = prefetch_rows_enabled() ? std::min<long long>(feat_bytes, 32ll << 20) / 128 : 0;
+  const long long feat_lines = std::min<long long>(feat_bytes, 32ll << 20) / 128;
+  const unsigned long long wait_limit_ns = test_wait_limit_us() > 0 ? (unsigned long long)test_wait_limit_us() * 1000ull : kWaitLimitNs;
+  const int withhold_first_w = test_wait_limit_us() > 0 ? 1 : 0;
 
   cudaLaunchConfig_t config = {};
   config.gridDim = dim3(unsigned(grid));
   config.blockDim = dim3(unsigned(C::kThreads));
-  config.dynamicSmemBytes = smem;
+  // Always the SM's whole shared memory, whatever the layout needs: one CTA per SM by construction.  The kernel
+  // allocates TMEM and lets its dependents start before it waits for its predecessors, so a second resident CTA (of
+  // this or of the next grid) could hold TMEM columns that a CTA waiting in tcgen05.alloc needs.
+  config.dynamicSmemBytes = kMaxSmem;
   config.stream = stream;
   cudaLaunchAttribute attribute[1];
   attribute[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see the kernel's griddepcontrol instructions
@@ -1162,7 +1177,8 @@ int launch(const void* feats, const void* w, const spconv_kmap* km, void* out, s
   SPCONV_CUDA_TRY(cudaLaunchKernelEx(&config, k_forward_tc<CIN, COUT, GROUPED>, wmap, static_cast<const uint8_t*>(feats), km->d.tile_nbr,
                                      km->d.tile_crow, km->d.tile_rows, km->d.tile_mask, km->d.tile_absent, km->d.sorted_tiles,
                                      static_cast<uint8_t*>(out), n_tiles, kvol, km->mask_words, G, rounds, cols, idesc,
-                                     dtype == SPCONV_BF16 ? 1 : 0, km->d.status, g_timeline, feat_lines, strict_order ? 1 : 0));
+                                     dtype == SPCONV_BF16 ? 1 : 0, km->d.status, g_timeline, feat_lines, strict_order ? 1 : 0, wait_limit_ns,
+                                     withhold_first_w));
   SPCONV_CUDA_TRY(cudaGetLastError());
   return SPCONV_OK;
 }
@@ -1184,6 +1200,8 @@ int dispatch_cout(const void* feats, const void* w, const spconv_kmap* km, void*
 }
 
 }  // namespace
+
+void set_forward_tc_test_wait_limit_us(long long us) { g_test_wait_limit_us.store(us > 0 ? us : 0, std::memory_order_relaxed); }
 
 // Diagnostics: install (or clear, with nullptr) a device buffer of 16 * gridDim uint64 that the
 // tensor-core kernel fills with per-CTA globaltimer stamps: 0 start, 1 set-up done, 2 step list built,

@@ -9,6 +9,7 @@
 #include <cub/device/device_radix_sort.cuh>
 
 #include <algorithm>
+#include <atomic>
 #include <chrono>
 #include <functional>
 #include <mutex>
@@ -698,14 +699,16 @@ k_sort_rows_coop(const int32_t* __restrict__ nbr, const int32_t* __restrict__ nb
     }
     grid.sync();
     {  // per digit: items of earlier blocks with this digit, and of all blocks.  Warp w sums the blocks b = w (mod 8);
-       // a lane takes eight consecutive digits of a block's counts as two vector loads, and the loads of up to
-       // twelve blocks are in flight together (one round trip for grids of up to 96 blocks).
+       // a lane takes eight consecutive digits of a block's counts as two vector loads, and the loads of several
+       // blocks are in flight together.
       before_s[tid] = 0u; total_s[tid] = 0u;
       __syncthreads();
       uint32_t bef[8], tot[8];
 #pragma unroll
       for (int j = 0; j < 8; ++j) { bef[j] = 0u; tot[j] = 0u; }
-      constexpr int kBatch = 12;
+      // (small grids: one round trip for up to 96 blocks; the instantiation for large grids keeps fewer loads in
+      // flight so that more of its blocks fit an SM, which is what bounds the rows a cooperative launch can take)
+      constexpr int kBatch = kSortItems <= kSortItemsSmall ? 12 : 4;
       for (unsigned b0 = warp; b0 < gridDim.x; b0 += kBatch * (kSortThreads / 32)) {
         uint4 c[kBatch][2];
 #pragma unroll
@@ -993,47 +996,71 @@ k_tile_plan_rows(const int32_t* __restrict__ tile_rows, const int32_t* __restric
   }
 }
 
-// Schedule of the tensor-core forward: tiles in descending order of their block count (counting sort by one
-// thread block), so that dealing them out serpentine over the CTAs gives every CTA nearly the same number
-// of blocks.  The order among tiles of equal count is arbitrary; it changes which CTA computes a tile, never
-// the values computed.
+// Schedule of the tensor-core forward: tiles in descending order of their block count, tiles of equal count in
+// ascending tile order (a stable counting sort by one thread block), so that dealing them out serpentine over the
+// CTAs gives every CTA nearly the same number of blocks and the same tiles on every run (the forward may
+// accumulate a CTA's heaviest tile in two parts, so which tiles share a CTA shows in the last bits of the result).
+// Thread i owns the contiguous chunk of tiles [i * chunk, (i + 1) * chunk).  Kernel volumes beyond 31 offsets
+// (more count classes than the per-thread counters hold) fall back to an unordered placement within a class.
 __device__ void schedule_tiles_block(const uint32_t* __restrict__ tile_mask, int n_tiles, int mask_words, int kvol,
                                      int32_t* __restrict__ sorted_tiles, uint32_t* __restrict__ status_words) {
-  __shared__ int hist[kMaskWordsMax * 32 + 2];
-  __shared__ int base[kMaskWordsMax * 32 + 2];
   if (threadIdx.x < 16) status_words[threadIdx.x] = 0u;   // the forward kernels' status record starts clean
-  for (int i = threadIdx.x; i <= kvol; i += blockDim.x) hist[i] = 0;
-  // Usual case (one mask word, at most kKeep tiles per thread): a thread reads its tiles' masks once, all reads
-  // in flight together, and keeps them in registers for both passes; this block runs alone at the end of the
-  // build, so its round trips to memory are the build's time.
-  constexpr int kKeep = 8;
-  if (mask_words == 1 && n_tiles <= kKeep * int(blockDim.x)) {
+  if (mask_words == 1 && kvol <= 31 && blockDim.x <= 128 && n_tiles <= 60000) {
+    constexpr int kClasses = 32, kMaxThreads = 128, kKeep = 8;
+    __shared__ uint16_t cnt[kClasses][kMaxThreads];   // tiles of class c in thread i's chunk, then their exclusive prefix over threads
+    __shared__ int class_base[kClasses];
+    const int T = int(blockDim.x), tid = int(threadIdx.x), lane = tid & 31, warp = tid >> 5;
+    const int chunk = (n_tiles + T - 1) / T;
+    const int beg = min(tid * chunk, n_tiles), end = min(beg + chunk, n_tiles);
+    for (int c = 0; c < kClasses; ++c) cnt[c][tid] = 0;
     uint32_t mine[kKeep];
 #pragma unroll
-    for (int i = 0; i < kKeep; ++i) {
-      const int t = int(threadIdx.x) + i * int(blockDim.x);
-      mine[i] = t < n_tiles ? __ldcg(tile_mask + t) : 0u;
-    }
-    __syncthreads();
+    for (int i = 0; i < kKeep; ++i) mine[i] = beg + i < end ? __ldcg(tile_mask + beg + i) : 0u;   // all reads in flight together
 #pragma unroll
-    for (int i = 0; i < kKeep; ++i)
-      if (int(threadIdx.x) + i * int(blockDim.x) < n_tiles) atomicAdd(&hist[__popc(mine[i])], 1);
+    for (int i = 0; i < kKeep; ++i) if (beg + i < end) cnt[__popc(mine[i])][tid] += 1;
+    for (int t = beg + kKeep; t < end; ++t) cnt[__popc(__ldcg(tile_mask + t))][tid] += 1;
     __syncthreads();
-    if (threadIdx.x == 0) {
+    // per class: exclusive prefix over the threads (warp w takes the classes w, w + nwarps, ...) and the class total
+    const int nwarps = (T + 31) / 32;
+    for (int c = warp; c < kClasses; c += nwarps) {
       int run = 0;
-      for (int c = kvol; c >= 0; --c) { base[c] = run; run += hist[c]; }
+      for (int i0 = 0; i0 < T; i0 += 32) {
+        const int i = i0 + lane;
+        const int v = i < T ? int(cnt[c][i]) : 0;
+        int incl = v;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) { const int u = __shfl_up_sync(0xffffffffu, incl, off); if (lane >= off) incl += u; }
+        if (i < T) cnt[c][i] = uint16_t(run + incl - v);
+        run += __shfl_sync(0xffffffffu, incl, 31);
+      }
+      if (lane == 0) class_base[c] = run;   // the total for now
     }
     __syncthreads();
-#pragma unroll
-    for (int i = 0; i < kKeep; ++i) {
-      const int t = int(threadIdx.x) + i * int(blockDim.x);
-      if (t >= n_tiles) continue;
-      int32_t* rec = sorted_tiles + size_t(atomicAdd(&base[__popc(mine[i])], 1)) * 2;
-      rec[0] = t;
-      rec[1] = int32_t(mine[i]);
+    if (tid == 0) {   // classes in descending order of their count value
+      int run = 0;
+      for (int c = kClasses - 1; c >= 0; --c) { const int total = class_base[c]; class_base[c] = run; run += total; }
     }
+    __syncthreads();
+    int placed[kClasses];
+#pragma unroll
+    for (int c = 0; c < kClasses; ++c) placed[c] = 0;
+    auto place = [&](int t, uint32_t m) {
+      const int c = __popc(m);
+      int mine_before = 0;
+#pragma unroll
+      for (int q = 0; q < kClasses; ++q) if (q == c) { mine_before = placed[q]; placed[q] += 1; }
+      int32_t* rec = sorted_tiles + size_t(class_base[c] + int(cnt[c][tid]) + mine_before) * 2;
+      rec[0] = t;
+      rec[1] = int32_t(m);
+    };
+#pragma unroll
+    for (int i = 0; i < kKeep; ++i) if (beg + i < end) place(beg + i, mine[i]);
+    for (int t = beg + kKeep; t < end; ++t) place(t, __ldcg(tile_mask + t));
     return;
   }
+  __shared__ int hist[kMaskWordsMax * 32 + 2];
+  __shared__ int base[kMaskWordsMax * 32 + 2];
+  for (int i = threadIdx.x; i <= kvol; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   for (int t = threadIdx.x; t < n_tiles; t += blockDim.x) {
     int c = 0;
@@ -1163,28 +1190,32 @@ int device_status_to_error(uint32_t st) {
   return SPCONV_OK;
 }
 
-// Number of blocks of the cooperative sort kernel that fit the device at once (0 if cooperative launches
-// are not supported).  An environment switch forces the library sort for testing.
-int coop_sort_capacity(int device) {
-  static int cap[64];
+// Number of blocks of the cooperative sort kernel that fit the device at once, for the instantiation with few items
+// per thread (large = false) and the one with many (0 if cooperative launches are not supported).  An environment
+// switch forces the library sort for testing.
+int coop_sort_capacity(int device, bool large) {
+  static int cap[64][2];
   static bool known[64] = {false};
   static std::mutex mu;
   if (device < 0 || device >= 64) return 0;
   std::lock_guard<std::mutex> lock(mu);
   if (!known[device]) {
-    int coop = 0, sms = 0, per_sm = 0;
+    int coop = 0, sms = 0, per_small = 0, per_large = 0;
     const char* off = std::getenv("SPCONV_KMAP_LIBRARY_SORT");
     if (!(off != nullptr && off[0] == '1') &&
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device) == cudaSuccess && coop != 0 &&
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess &&
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_sort_rows_coop<kSortItemsLarge>, kSortThreads, 0) == cudaSuccess)
-      cap[device] = sms * per_sm;
-    else
-      cap[device] = 0;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_small, k_sort_rows_coop<kSortItemsSmall>, kSortThreads, 0) == cudaSuccess &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_large, k_sort_rows_coop<kSortItemsLarge>, kSortThreads, 0) == cudaSuccess) {
+      cap[device][0] = sms * per_small;
+      cap[device][1] = sms * per_large;
+    } else {
+      cap[device][0] = cap[device][1] = 0;
+    }
     (void)cudaGetLastError();
     known[device] = true;
   }
-  return cap[device];
+  return cap[device][large ? 1 : 0];
 }
 
 
@@ -1199,7 +1230,11 @@ int max_candidates_per_axis(int K, int s, int d) {
   return best;
 }
 
+std::atomic<long long> g_test_table_slots{0};
+
 }  // namespace
+
+void set_kmap_test_table_slots(long long slots) { g_test_table_slots.store(slots > 0 ? slots : 0, std::memory_order_relaxed); }
 
 void destroy_kmap_impl(spconv_kmap* km) {
   if (!km) return;
@@ -1281,10 +1316,12 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
 
   const int nblk = int((nq + kBlock - 1) / kBlock);
   const int64_t M = int64_t(nblk) * kvol;
-  // Load factor of the location table: at most 1/kTableSlack.  Probe sequences are walked by whole warps (a warp
-  // takes as many rounds as its unluckiest lane), so short sequences matter more than the table's size.
-  static const int kTableSlack = [] { const char* e = std::getenv("SPCONV_KMAP_TABLE_SLACK"); return e != nullptr ? std::max(2, std::atoi(e)) : 4; }();
-  const uint32_t cap1 = pow2_at_least(uint64_t(kTableSlack) * std::max<int64_t>(n, 1));
+  // Load factor of the location table: at most 1/4.  Probe sequences are walked by whole warps (a warp takes as
+  // many rounds as its unluckiest lane), so short sequences matter more than the table's size.
+  // Test hook (spconv_test_hook, SPCONV_HOOK_TABLE_SLOTS): a positive value forces the table to pow2(value) slots
+  // whatever the input, so that a test can make the bounded probe sequence run out (SPCONV_ERR_TABLE_FULL).
+  const long long forced_slots = g_test_table_slots.load(std::memory_order_relaxed);
+  const uint32_t cap1 = forced_slots > 0 ? pow2_at_least(uint64_t(forced_slots)) : pow2_at_least(uint64_t(4) * std::max<int64_t>(n, 1));
   const dim3 grid_kn(nblk, kvol);
   const int4* coords4 = reinterpret_cast<const int4*>(coords);
   const int4* qcoords4 = inverse ? reinterpret_cast<const int4*>(fine_coords) : coords4;
@@ -1403,15 +1440,16 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
       uint32_t* rkeys_sorted = ta.take<uint32_t>(no);
       int32_t* rrows = ta.take<int32_t>(no);
       int32_t* rrows_b = ta.take<int32_t>(no);
+      // few items per thread while all such blocks (and the scan's block) are resident at once, else many
       const int small_blocks = int((padded + kSortThreads * kSortItemsSmall - 1) / (kSortThreads * kSortItemsSmall));
-      const bool small_sort = small_blocks <= kSortSmallMaxBlocks;
+      const bool small_sort = small_blocks <= kSortSmallMaxBlocks && small_blocks + 1 <= coop_sort_capacity(km->device, false);
       const int sort_tile = kSortThreads * (small_sort ? kSortItemsSmall : kSortItemsLarge);
       const int sort_blocks = int((padded + sort_tile - 1) / sort_tile);
       uint32_t* block_hist = ta.take<uint32_t>(size_t(sort_blocks + 1) * 256);
       void* cub_tmp = ta.take<char>(cub_tmp_bytes);
       size_t tmp_bytes = cub_tmp_bytes;
       const unsigned* order_cnt = (scan_pending || counts_based) ? d_offset_cnt : nullptr;   // the probe's per-offset totals order the key bits
-      if (sort_blocks + 1 <= coop_sort_capacity(km->device)) {
+      if (sort_blocks + 1 <= coop_sort_capacity(km->device, !small_sort)) {
         // every block resident at once: keys and all sort passes in one cooperative launch
         const int32_t* nbr_arg = km->d.nbr;
         const int32_t* rows_arg = plan_rows;

@@ -31,6 +31,19 @@ def test_simt_kernel_small(dtype, cin, cout):
     check_layer(coords, _layer("spconv", 3, 2, cin, cout, dtype), algo="simt")
 
 
+@pytest.mark.parametrize("cin,cout,K", [(16, 16, 3), (32, 32, 3), (16, 16, 5), (12, 20, 3), (4, 4, 1), (16, 64, 2)])
+def test_fp32_weights_resident_kernel(cin, cout, K):
+    """fp32 layers whose weights fit shared memory take the kernel that stages all of them once (more than 48 KB for
+    32 -> 32, K = 3 and for K = 5): submanifold and strided maps, channel counts that do not divide a warp, every
+    row checked at the fp32 tolerance, and the result must not depend on the neighbours of a block (ragged tail)."""
+    coords = wl.shuffle_rows(wl.random_blob(2100, 15, 9, batches=2), seed=8)
+    if K % 2 == 1:
+        km, y = check_layer(coords, _layer("subm", K, 1, cin, cout, "f32"), algo="simt")
+        _, y_auto = check_layer(coords, _layer("subm", K, 1, cin, cout, "f32"), km=km)
+        assert torch.equal(y, y_auto)            # fp32 always runs on the CUDA-core path
+    check_layer(coords, _layer("spconv", K, 2, cin, cout, "f32"), algo="simt")
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f16"])
 @pytest.mark.parametrize("cin", [16, 32, 64, 128])
 @pytest.mark.parametrize("cout", [16, 32, 64, 128])
