@@ -139,6 +139,26 @@ int spconv_build_kmap(const int32_t* coords, int64_t n, int stride, int dilation
 int spconv_build_inverse_kmap(const int32_t* fine_coords, int64_t n_fine, const int32_t* coarse_coords, int64_t n_coarse,
                               int stride, int dilation, int kernel_size, void* cuda_stream, spconv_kmap_t** kmap_out);
 
+/*
+ * Submanifold kernel map with the location table as a DENSE ARRAY over a stated grid instead of the hash table.
+ * [Sec. III-C.1: "we can also use a three-dimensional array as location table", the variant the paper prefers
+ * where the domain is confined; the printed createLCTKernel stores the row index at the cell's linear index, Eq. 6]
+ *
+ *   coords, n, dilation, cuda_stream, kmap_out   as for spconv_build_kmap with stride 1, submanifold 1.
+ *   grid_shape    HOST int32[4] = (B, X, Y, Z): every input row must satisfy 0 <= b < B, 0 <= x < X, 0 <= y < Y,
+ *                 0 <= z < Z (else SPCONV_ERR_COORD_RANGE); B*X*Y*Z <= SPCONV_DENSE_MAX_CELLS (else
+ *                 SPCONV_ERR_TOO_LARGE): one int32 per cell is filled and probed per build (16 MiB at the limit).
+ *   kernel_size   1 or 3.
+ * The cell of (b, x, y, z) is ((b*X + x)*Y + y)*Z + z (the batch index is part of the address; Eq. 6 has none).
+ * The resulting handle is indistinguishable from spconv_build_kmap's: same row numbering, offset table, pair
+ * lists and tile plan, bit for bit.  Duplicates are detected as there.  Which of the two builds faster depends on
+ * the grid's volume against the number of rows: the array costs its fill, the hash table its probing.
+ * Errors: INVALID_ARG, TOO_LARGE, COORD_RANGE, DUPLICATE_COORD, ALLOC, CUDA.
+ */
+#define SPCONV_DENSE_MAX_CELLS 4194304
+int spconv_build_kmap_dense(const int32_t* coords, int64_t n, const int32_t* grid_shape /* host [4] */, int dilation,
+                            int kernel_size, void* cuda_stream, spconv_kmap_t** kmap_out);
+
 /* Describe a kernel map.  `info` is host memory; the pointers inside stay valid until destroy. */
 int spconv_kmap_info(const spconv_kmap_t* kmap, spconv_kmap_info_t* info);
 

@@ -21,7 +21,7 @@ _TORCH_DTYPE = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
 DTYPE_BY_NAME = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
 
 EXPORTS = (
-    "spconv_build_kmap", "spconv_build_inverse_kmap", "spconv_kmap_info", "spconv_kmap_destroy", "spconv_forward", "spconv_forward_algo",
+    "spconv_build_kmap", "spconv_build_inverse_kmap", "spconv_build_kmap_dense", "spconv_kmap_info", "spconv_kmap_destroy", "spconv_forward", "spconv_forward_algo",
     "spconv_last_device_status", "spconv_layer", "spconv_layer_host", "spconv_strerror", "spconv_subm_offset_table_noalloc",
     "spconv_kmap_status_words", "spconv_test_hook",
 )
@@ -65,6 +65,8 @@ def load() -> ctypes.CDLL:
         lib.spconv_build_kmap.argtypes = [vp, i64, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
         lib.spconv_build_inverse_kmap.restype = i32
         lib.spconv_build_inverse_kmap.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        lib.spconv_build_kmap_dense.restype = i32
+        lib.spconv_build_kmap_dense.argtypes = [vp, i64, ctypes.POINTER(ctypes.c_int32), i32, i32, vp, ctypes.POINTER(vp)]
         lib.spconv_kmap_info.restype = i32
         lib.spconv_kmap_info.argtypes = [vp, ctypes.POINTER(_KmapInfo)]
         lib.spconv_kmap_destroy.restype = None
@@ -191,6 +193,20 @@ def spconv_build_kmap(coords: torch.Tensor, stride: int = 1, dilation: int = 1, 
                                   ctypes.c_void_p(_stream_ptr(stream)), ctypes.byref(h))
     if st != 0:
         raise SpconvError(st, "spconv_build_kmap")
+    return Kmap(h.value)
+
+
+def spconv_build_kmap_dense(coords: torch.Tensor, grid_shape, dilation: int = 1, kernel_size: int = 3, stream=None) -> Kmap:
+    """Submanifold kernel map built through a dense-array location table over ``grid_shape = (B, X, Y, Z)``."""
+    if not (coords.is_cuda and coords.dtype == torch.int32 and coords.dim() == 2 and coords.shape[1] == 4
+            and coords.is_contiguous()):
+        raise ValueError("coords must be a contiguous CUDA int32 tensor of shape [n, 4]")
+    shape = (ctypes.c_int32 * 4)(*[int(v) for v in grid_shape])
+    h = ctypes.c_void_p(None)
+    st = load().spconv_build_kmap_dense(ctypes.c_void_p(coords.data_ptr() if coords.numel() else 0), coords.shape[0], shape,
+                                        int(dilation), int(kernel_size), ctypes.c_void_p(_stream_ptr(stream)), ctypes.byref(h))
+    if st != 0:
+        raise SpconvError(st, "spconv_build_kmap_dense")
     return Kmap(h.value)
 
 

@@ -66,6 +66,26 @@ int spconv_build_inverse_kmap(const int32_t* fine_coords, int64_t n_fine, const 
                          nullptr, fine_coords != nullptr ? fine_coords : none, n_fine);
 }
 
+int spconv_build_kmap_dense(const int32_t* coords, int64_t n, const int32_t* grid_shape, int dilation, int kernel_size,
+                            void* cuda_stream, spconv_kmap_t** kmap_out) {
+  if (kmap_out == nullptr) return SPCONV_ERR_INVALID_ARG;
+  *kmap_out = nullptr;
+  if (n < 0 || dilation < 1 || dilation > 4096 || grid_shape == nullptr) return SPCONV_ERR_INVALID_ARG;
+  if (kernel_size != 1 && kernel_size != 3) return SPCONV_ERR_INVALID_ARG;
+  if (n > 0 && coords == nullptr) return SPCONV_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(coords) & 15u) return SPCONV_ERR_INVALID_ARG;
+  int grid[4];
+  int64_t cells = 1;
+  for (int a = 0; a < 4; ++a) {
+    if (grid_shape[a] < 1 || grid_shape[a] > 65535) return SPCONV_ERR_INVALID_ARG;
+    grid[a] = grid_shape[a];
+    cells *= grid_shape[a];
+    if (cells > int64_t(SPCONV_DENSE_MAX_CELLS)) return SPCONV_ERR_TOO_LARGE;
+  }
+  if (n * int64_t(kernel_size) * kernel_size * kernel_size > int64_t(2000000000)) return SPCONV_ERR_TOO_LARGE;
+  return build_kmap_impl(coords, n, 1, dilation, kernel_size, 1, static_cast<cudaStream_t>(cuda_stream), kmap_out, nullptr, nullptr, 0, grid);
+}
+
 int spconv_kmap_info(const spconv_kmap_t* km, spconv_kmap_info_t* info) {
   if (km == nullptr || info == nullptr) return SPCONV_ERR_INVALID_ARG;
   std::memset(info, 0, sizeof(*info));

@@ -61,7 +61,9 @@ namespace spconv {
 // (rows of the input features), fine_coords [n_fine][4] the output rows, and submanifold must be 0.
 int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, int kernel, int submanifold,
                     cudaStream_t stream, spconv_kmap** out, const std::function<int(spconv_kmap*)>* before_wait = nullptr,
-                    const int32_t* fine_coords = nullptr, int64_t n_fine = 0);
+                    const int32_t* fine_coords = nullptr, int64_t n_fine = 0, const int* dense_grid = nullptr);
+// dense_grid (optional, host int[4] = B, X, Y, Z): the location table is a dense array over that grid instead of the
+// hash table (submanifold maps with kernel size 1 or 3 only; the caller checks the shape and its size).
 void destroy_kmap_impl(spconv_kmap* km);
 void set_kmap_test_table_slots(long long slots);          // test hook, see spconv_test_hook
 

@@ -196,6 +196,32 @@ __global__ void k_subm_probe(const int4* __restrict__ coords, int n, int K, int 
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Location table as a dense array over a stated grid (Sec. III-C.1: "a three-dimensional array as location
+// table", the alternative the paper prefers where the domain is confined): cell (b, x, y, z) of a B x X x Y x Z
+// grid holds the input row at that position or -1, at index ((b*X + x)*Y + y)*Z + z (z fastest, as the rows of a
+// sorted input and the kernel offsets run).  A lookup is one read at a computed address, without hashing or
+// probing; neighbouring positions are neighbouring words.
+struct GridDims { int b, x, y, z; };
+__device__ __forceinline__ bool in_grid(const GridDims& g, int b, int x, int y, int z) {
+  return uint32_t(b) < uint32_t(g.b) && uint32_t(x) < uint32_t(g.x) && uint32_t(y) < uint32_t(g.y) && uint32_t(z) < uint32_t(g.z);
+}
+__device__ __forceinline__ size_t grid_cell(const GridDims& g, int b, int x, int y, int z) {
+  return ((size_t(b) * g.x + x) * g.y + y) * g.z + z;
+}
+// One thread per input row, like the paper's createLCTKernel, with the batch index in the cell address and the
+// two checks the printed kernel lacks: positions outside the grid and duplicates are reported.
+__global__ void k_insert_dense(const int4* __restrict__ coords, int n, int32_t* __restrict__ cells, const __grid_constant__ GridDims grid,
+                               uint32_t* status) {
+  chain_begin();
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int4 c = coords[i];
+  if (!in_grid(grid, c.x, c.y, c.z, c.w)) { atomicOr(status, kDevCoordRange); return; }
+  if (atomicCAS(cells + grid_cell(grid, c.x, c.y, c.z, c.w), -1, i) != -1) atomicOr(status, kDevDuplicate);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Offset table, every offset of one output row per thread (kernel volumes up to 32).
 //   MODE 0, submanifold (Sec. III-C.2): row j looks at p_j + d*(kvec - r); the centre offset is j itself.
@@ -207,12 +233,15 @@ __global__ void k_subm_probe(const int4* __restrict__ coords, int n, int K, int 
 // nbr_rows[j][k] (the paper's OFT layout; the tile plan reads whole rows of permuted j).  row_mask[j] has bit k
 // set where the row has an input through offset k.  Per block and offset the number of hits goes to blockcnt
 // (the pair emission's bases), per offset the total to offset_cnt.
-template <int K, int MODE>
+// DENSE: the location table is the dense array of k_insert_dense (`table` then points at its cells and `grid`
+// gives its shape): every offset's cell is read directly, all reads in flight together, and there is no filter.
+template <int K, int MODE, bool DENSE = false>
 __global__ void __launch_bounds__(kBlock)
 k_probe_rows(const int4* __restrict__ qcoords, int nq, int dil, int stride, const LocSlot* __restrict__ table,
              uint32_t capmask, const uint32_t* __restrict__ occ, int32_t* __restrict__ nbr,
              int32_t* __restrict__ nbr_rows, uint32_t* __restrict__ row_mask, int32_t* __restrict__ blockcnt,
-             unsigned* __restrict__ offset_cnt, int4* __restrict__ coords_copy, uint32_t* __restrict__ status) {
+             unsigned* __restrict__ offset_cnt, int4* __restrict__ coords_copy, uint32_t* __restrict__ status,
+             const __grid_constant__ GridDims grid) {
   chain_begin();
   SPCONV_TL(2);
   constexpr int KV = K * K * K;
@@ -252,7 +281,18 @@ k_probe_rows(const int4* __restrict__ qcoords, int nq, int dil, int stride, cons
   };
   // 1. candidates: offsets whose position the occupancy filter does not rule out (all reads in flight together)
   uint32_t cand = 0u;
-  {
+  if constexpr (DENSE) {
+    const int32_t* cells = reinterpret_cast<const int32_t*>(table);
+    int got[KV];
+#pragma unroll
+    for (int k = 0; k < KV; ++k) {
+      int x, y, z;
+      const bool valid = target(k, x, y, z) && in_grid(grid, c.x, x, y, z);
+      got[k] = valid ? __ldg(cells + grid_cell(grid, c.x, x, y, z)) : -1;
+    }
+#pragma unroll
+    for (int k = 0; k < KV; ++k) s_v[k][tid] = (MODE == 0 && k == (r * K + r) * K + r && live) ? j : got[k];
+  } else {
     uint32_t word[KV];
 #pragma unroll
     for (int k = 0; k < KV; ++k) {
@@ -1282,7 +1322,7 @@ struct TimelineDump {
 
 int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, int kernel, int submanifold,
                     cudaStream_t stream, spconv_kmap** out, const std::function<int(spconv_kmap*)>* before_wait,
-                    const int32_t* fine_coords, int64_t n_fine) {
+                    const int32_t* fine_coords, int64_t n_fine, const int* dense_grid) {
   [[maybe_unused]] StageTimer stages(stream);
 #ifdef SPCONV_KMAP_TIMELINE
   TimelineDump timeline_dump{stream};
@@ -1357,7 +1397,8 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     return pad256(*cub_bytes) + pad256(size_t(items) * 4) * 4 + pad256((size_t(items) / (kSortThreads * kSortItemsSmall) + 8) * 1024) + 1024;
   };
   size_t cub_bytes = 0;
-  size_t scratch_bytes = pad256(size_t(cap1) * sizeof(LocSlot)) + pad256(size_t(kOccWords) * 4) + pad256(size_t(M) * 4) * 2 +
+  size_t scratch_bytes = pad256(std::max(size_t(cap1) * sizeof(LocSlot), dense_grid != nullptr ? size_t(dense_grid[0]) * dense_grid[1] * dense_grid[2] * dense_grid[3] * 4 : size_t(0))) +
+                         pad256(size_t(kOccWords) * 4) + pad256(size_t(M) * 4) * 2 +
                          pad256(size_t(M) * 8) * 2 + pad256((size_t(kvol) + 1 + 8 + 16) * 8) + pad256(32) + 4096;
   if (known_outputs) scratch_bytes += sort_bytes_for(nq, &cub_bytes);   // n_out is known: the sort's buffers ride along
   if (known_outputs && rows_table) scratch_bytes += pad256(size_t(nq) * 128) + pad256(size_t(nq) * 4);
@@ -1367,10 +1408,16 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   scratch.stream = stream;
   SPCONV_CUDA_TRY(cudaMallocAsync(&scratch.ptr, scratch_bytes, stream));
   Arena sa{static_cast<char*>(scratch.ptr), scratch_bytes, 0};
-  LocSlot* table1 = sa.take<LocSlot>(cap1);
-  // the occupancy filter lies right behind the table: one fill empties both
-  uint32_t* occ = (known_outputs && rows_table) ? sa.take<uint32_t>(kOccWords) : nullptr;
-  const size_t table_fill_bytes = occ != nullptr ? size_t(reinterpret_cast<char*>(occ + kOccWords) - reinterpret_cast<char*>(table1)) : size_t(cap1) * sizeof(LocSlot);
+  // Location table: the hash table with its occupancy filter right behind it (one fill empties both), or, where the
+  // caller stated a grid, the dense array of that grid's cells (every byte 0xFF = -1: no row).
+  GridDims grid_dims{0, 0, 0, 0};
+  if (dense_grid != nullptr) grid_dims = GridDims{dense_grid[0], dense_grid[1], dense_grid[2], dense_grid[3]};
+  const size_t dense_cells = dense_grid != nullptr ? size_t(dense_grid[0]) * dense_grid[1] * dense_grid[2] * dense_grid[3] : 0;
+  LocSlot* table1 = dense_grid != nullptr ? reinterpret_cast<LocSlot*>(sa.take<int32_t>(dense_cells)) : sa.take<LocSlot>(cap1);
+  uint32_t* occ = (known_outputs && rows_table && dense_grid == nullptr) ? sa.take<uint32_t>(kOccWords) : nullptr;
+  const size_t table_fill_bytes = dense_grid != nullptr ? dense_cells * 4
+                                  : occ != nullptr ? size_t(reinterpret_cast<char*>(occ + kOccWords) - reinterpret_cast<char*>(table1))
+                                                   : size_t(cap1) * sizeof(LocSlot);
   int32_t* cnt_a = sa.take<int32_t>(M);
   int32_t* cnt_b = sa.take<int32_t>(M);
   int64_t* excl_a = sa.take<int64_t>(M);
@@ -1555,7 +1602,10 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     SPCONV_STAGE(stages, "alloc+memset");
     SPCONV_HOST_TL("allocs+memsets");
     int4* out_coords4 = reinterpret_cast<int4*>(km->d.out_coords);
-    if (n > 0)
+    if (n > 0 && dense_grid != nullptr)
+      SPCONV_CUDA_TRY(launch_chained(k_insert_dense, dim3(nblk_in), dim3(kBlock), stream, coords4, int(n), reinterpret_cast<int32_t*>(table1),
+                                     grid_dims, d_status));
+    else if (n > 0)
       SPCONV_CUDA_TRY(launch_chained(k_insert, dim3(nblk_in), dim3(kBlock), stream, coords4, int(n), table1, cap1 - 1, d_status,
                                      (submanifold && !rows_table) ? out_coords4 : static_cast<int4*>(nullptr), occ));
     SPCONV_STAGE(stages, "insert");
@@ -1564,10 +1614,11 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
       auto probe_rows = [&](auto kernel) {
         return launch_chained(kernel, dim3(nblk), dim3(kBlock), stream, qcoords4, int(nq), d, s, static_cast<const LocSlot*>(table1),
                               cap1 - 1, static_cast<const uint32_t*>(occ), km->d.nbr, nbr_rows, row_mask,
-                              cnt_a, d_offset_cnt, out_coords4, d_status);
+                              cnt_a, d_offset_cnt, out_coords4, d_status, grid_dims);
       };
       cudaError_t le = cudaErrorInvalidValue;
-      if (!inverse) le = K == 1 ? probe_rows(k_probe_rows<1, 0>) : probe_rows(k_probe_rows<3, 0>);
+      if (dense_grid != nullptr) le = K == 1 ? probe_rows(k_probe_rows<1, 0, true>) : probe_rows(k_probe_rows<3, 0, true>);
+      else if (!inverse) le = K == 1 ? probe_rows(k_probe_rows<1, 0>) : probe_rows(k_probe_rows<3, 0>);
       else le = K == 1 ? probe_rows(k_probe_rows<1, 1>) : K == 2 ? probe_rows(k_probe_rows<2, 1>) : probe_rows(k_probe_rows<3, 1>);
       SPCONV_CUDA_TRY(le);
       plan_rows = nbr_rows;
