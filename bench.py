@@ -11,8 +11,9 @@ rotates over eight different sweeps, whose arrays together are about three times
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-N > 1 is launched by torchrun, one rank per GPU; each rank processes its own sweep (seed = rank), no
-data-path collective (sweeps are independent: coordinates with different batch indices never pair).
+N > 1 runs one rank per GPU under torchrun (started by the caller, or by this script itself when it is run
+plainly with --gpus N); each rank processes its own sweeps (seed = rank), no data-path collective (sweeps are
+independent: coordinates with different batch indices never pair).
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
 """
 from __future__ import annotations
@@ -40,12 +41,15 @@ CIN = COUT = 64
 KVOL = 27
 DTYPE = "bf16"
 REFERENCE_SAMPLE_VOXELS = 10**9   # the oracle finishes the whole sweep in a fraction of a second: no sub-sampling
-# DRAM bytes (read + write) of one forward launch on this workload, from the ncu capture summarised in
-# profiles/forward_tc_config3_ncu.md (dram__bytes_read.sum + dram__bytes_write.sum, L2 flushed by ncu).
+# DRAM bytes (read + write) of one forward launch on sweep 0, from one profiler capture of this kernel
+# (dram__bytes_read.sum + dram__bytes_write.sum with the profiler's cache flush before the launch).  It is a
+# recorded figure, not measured by this script: the line says so in `traffic_source`.
 FORWARD_DRAM_TRAFFIC_BYTES = 15_232_512
-# Our kernels launched per step: k_insert, k_subm_probe, k_sort_rows_coop (row keys + radix sort + count scan,
-# one cooperative launch), k_tile_plan (its last block also orders the tiles), k_subm_emit (kernel-map build)
-# + k_forward_tc.
+FORWARD_DRAM_TRAFFIC_SOURCE = ("one profiler capture of k_forward_tc<64,64> on sweep 0 (DRAM bytes read + written per launch, "
+                               "caches flushed before the launch); recorded, not measured in this run")
+# Our kernels launched per step: k_insert, k_probe_rows (every offset of a row per thread), k_subm_emit (on a second
+# stream), k_sort_rows_coop (row keys + radix sort, one cooperative launch), k_tile_plan_rows (its last block also
+# orders the tiles and reports to the host) for the kernel map, + k_forward_tc.
 OUR_LAUNCHES_PER_STEP = 6
 ROTATION = 8   # sweeps a rank rotates over (about 45 MB of arrays each)
 
@@ -56,6 +60,13 @@ def measured_peaks():
         p = json.load(open(path))
         return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]), source="measured")
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+
+
+def kmap_algorithmic_bytes(n, pairs):
+    """Compulsory bytes of one submanifold kernel-map build: read the coordinates (16 B per row), fill and write a
+    location table of two slots of 12 bytes per row (keys + rows), write the offset table (4 * K^3 B per row) and
+    the pair lists (8 B per pair)."""
+    return n * (16 + 2 * 2 * 12 + 4 * KVOL) + 8 * pairs
 
 
 def forward_algorithmic_bytes(n_in, n_out, pairs):
@@ -385,7 +396,8 @@ def run_ours(args):
         pk.close()
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": total_ms_max / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": total_ms_max / args.steps, "ms_per_step_min": min(step_ms), "ms_per_step_median": statistics.median(step_ms),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "n_voxels": n, "pairs": int(pairs), "tiles": int(n_tiles),
                        "tile_blocks": int(blocks), "seed": seed,
@@ -398,12 +410,20 @@ def run_ours(args):
                       "forward_ms_flushed_single_launch": statistics.mean(fwd_ms),
                       "forward_ms_l2_warm": fwd_warm_ms,
                       "eff_tflops_l2_cold": flops / (fwd * 1e-3) / 1e12, "eff_tflops_l2_warm": flops / (fwd_warm_ms * 1e-3) / 1e12,
+                      "kmap_build_ms_min": min(kmap_ms), "kmap_build_ms_median": statistics.median(kmap_ms),
                       "kmap_build_mvoxels_s": rot_n / (statistics.mean(kmap_ms) * 1e-3) / 1e6,
+                      "kmap_algorithmic_bytes": kmap_algorithmic_bytes(rot_n, rot_pairs_mean),
+                      "kmap_roofline_frac": kmap_algorithmic_bytes(rot_n, rot_pairs_mean) / (peaks["hbm_gbs"] * 1e9) / (statistics.mean(kmap_ms) * 1e-3),
+                      "kmap_share_of_step": statistics.mean(kmap_ms) / statistics.mean(two_call_ms),
                       "t_hbm_us": t_hbm_us, "t_mma_us": t_mma_us,
                       "roofline_frac_l2_cold": max(t_hbm_us, t_mma_us) / (fwd * 1e3),
                       "roofline_frac_l2_warm": max(t_hbm_us, t_mma_us) / (fwd_warm_ms * 1e3)},
             "roofline": {"kernel": "k_forward_tc<64,64>", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
                          "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": FORWARD_DRAM_TRAFFIC_BYTES,
+                         "traffic_source": FORWARD_DRAM_TRAFFIC_SOURCE,
+                         "frac_single_launch_after_flush": alg_bytes / (statistics.mean(fwd_ms) * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                         "frac_note": "frac uses the period of back-to-back launches over rotating (L2-cold) sweeps, where a launch's set-up overlaps "
+                                      "the tail of the launch before; frac_single_launch_after_flush is one isolated launch",
                          "peak_source": peaks["source"], "algorithmic_bytes": alg_bytes, "ms": fwd},
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms_max, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h},
@@ -482,6 +502,19 @@ def run_survey(args):
     print(json.dumps({"survey": rows, "peaks": peaks}))
 
 
+def respawn_under_torchrun(args):
+    """`python bench.py --gpus N` with N > 1 and no launcher around it: start the N ranks here (one per GPU, NCCL
+    rendezvous on 127.0.0.1) and pass their output through."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__), "--gpus", str(args.gpus), "--steps", str(args.steps),
+           "--warmup", str(args.warmup), "--impl", args.impl]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -492,6 +525,8 @@ def main():
                     help="run three launches of one stage and exit (for profiler captures)")
     ap.add_argument("--survey", action="store_true", help="per-layer table over all five workloads (one JSON line)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.survey and not args.only:
+        sys.exit(respawn_under_torchrun(args))
     if args.survey:
         run_survey(args)
     elif args.impl == "reference":

@@ -43,38 +43,14 @@
 namespace spconv {
 namespace {
 
-#ifndef SPCONV_TC_PIPES
-#define SPCONV_TC_PIPES 2
-#endif
-constexpr int kMaxPipes = SPCONV_TC_PIPES;       // independent gather -> MMA pipelines per CTA (fewer when the A ring is short)
-#ifndef SPCONV_TC_GROUP_WARPS
-#define SPCONV_TC_GROUP_WARPS 8
-#endif
-constexpr int kGroupWarps = SPCONV_TC_GROUP_WARPS;   // producer warps of one pipeline (they share a step's rows)
+constexpr int kMaxPipes = 2;                     // independent gather -> MMA pipelines per CTA (fewer when the A ring is short)
+constexpr int kGroupWarps = 8;                   // producer warps of one pipeline (they share a step's rows)
 constexpr int kGroupThreads = 32 * kGroupWarps;
-#ifndef SPCONV_TC_ASTAGES
-#define SPCONV_TC_ASTAGES 12
-#endif
-#ifndef SPCONV_TC_WSTAGES
-#define SPCONV_TC_WSTAGES 4
-#endif
-#ifndef SPCONV_TC_W_IN_STAGE
-#define SPCONV_TC_W_IN_STAGE 1
-#endif
-#ifndef SPCONV_TC_IN_STAGE_MIN
-#define SPCONV_TC_IN_STAGE_MIN 3
-#endif
-#ifndef SPCONV_TC_GROUPED
-#define SPCONV_TC_GROUPED 1
-#endif
-#ifndef SPCONV_TC_GROUPED_MAX_CIN
-#define SPCONV_TC_GROUPED_MAX_CIN 64
-#endif
-constexpr int kGroupMaxCin = SPCONV_TC_GROUPED_MAX_CIN;   // widest input rows that take several offsets per step
-constexpr bool kGroupSteps = SPCONV_TC_GROUPED != 0;
+constexpr int kMaxAStages = 12;                  // most stages a CTA's rings hold in all
+constexpr int kInStageMin = 3;                   // a stage carries its W_k where at least this many stages per pipeline fit
+constexpr int kGroupMaxCin = 64;                 // widest input rows that take several offsets per step
 // Shapes that take several offsets per step: short rows always; 128-byte rows (two offsets) only where two such stages per pipeline fit.
-constexpr bool grouped_shape(int cin, int cout) { return kGroupSteps && cin <= kGroupMaxCin && (cin < 64 || cout <= 64); }   // (64 channels in: two panels must fit)   // steps of up to 128 / row bytes offsets for rows shorter than 128 bytes
-constexpr int kMaxAStages = SPCONV_TC_ASTAGES;
+constexpr bool grouped_shape(int cin, int cout) { return cin <= kGroupMaxCin && (cin < 64 || cout <= 64); }
 constexpr int kMaxGroup = 32;                    // tiles a CTA keeps in TMEM at once (<= 512 / COUT)
 constexpr uint32_t kSpinLimit = 1u << 24;        // polls per wait, and
 constexpr uint64_t kWaitLimitNs = 250ull * 1000 * 1000;  // wall-time bound per wait (0.25 s) unless a test shortens it
@@ -123,8 +99,8 @@ struct Cfg {
   // wait for and release (kSharedW); and if even that does not fit there is one pipeline.
   static constexpr int kAvail = kMaxSmem - 1024 - 12 * 1024;
   static constexpr int kInStageFit = kAvail / (kABytes + kWSlotBytes);
-  static constexpr bool kWInStage = SPCONV_TC_W_IN_STAGE != 0 && kMaxPipes > 1 && kInStageFit / kMaxPipes >= (GROUPED ? 2 : SPCONV_TC_IN_STAGE_MIN);
-  static constexpr int kWSlotsPrivate = kWBytes >= 16384 ? 2 : (kWBytes >= 8192 ? 3 : SPCONV_TC_WSTAGES);
+  static constexpr bool kWInStage = kMaxPipes > 1 && kInStageFit / kMaxPipes >= (GROUPED ? 2 : kInStageMin);
+  static constexpr int kWSlotsPrivate = kWBytes >= 16384 ? 2 : (kWBytes >= 8192 ? 3 : 4);
   static constexpr int kWSlotsShared = kWBytes >= 32768 ? 2 : 4;
   static constexpr bool kPrivateFits = kWInStage || kMaxPipes * (kWSlotsPrivate * kWSlotBytes + 2 * kABytes) <= kAvail;
   static constexpr bool kSharedW = !kPrivateFits && kMaxPipes > 1 && kMaxPipes * 2 * kABytes + kWSlotsShared * kWSlotBytes <= kAvail;

@@ -308,10 +308,7 @@ k_probe_rows(const int4* __restrict__ qcoords, int nq, int dil, int stride, cons
   }
   // 2. the candidates' table lookups, four at a time
   while (cand != 0u) {
-#ifndef SPCONV_PROBE_BATCH
-#define SPCONV_PROBE_BATCH 4
-#endif
-    constexpr int B = SPCONV_PROBE_BATCH;
+    constexpr int B = 4;
     int kk[B];
     uint64_t key[B];
     LocSlot got[B];
