@@ -252,7 +252,7 @@ int spconv_layer_host(const int32_t* coords_host, int64_t n, const void* feats_h
  * own allocator (an inference-engine plug-in's enqueue call is the typical case), or a control loop with
  * a memory budget fixed at start-up, where a cudaMalloc could fail, would stall the device, or is simply
  * forbidden.  spconv_build_kmap sizes and allocates its hash table per call; this entry point instead
- * probes a hash table kept in a fixed array inside the library (about 3 MiB, held by every GPU that loads
+ * probes a hash table kept in a fixed array inside the library (about 4 MiB, held by every GPU that loads
  * the library until the process exits) and writes straight into the caller's buffer.  It calls no
  * cudaMalloc / cudaFree, no stream-ordered allocator and no allocating library routine.  (The array is part
  * of the library's device code: the driver reserves it when it loads that code on a GPU, which with lazy
