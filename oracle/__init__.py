@@ -147,3 +147,50 @@ def forward(feats, w, oft) -> np.ndarray:
 def num_threads() -> int:
     """Threads the forward loop uses (OpenMP default for this host)."""
     return int(_load().oracle_num_threads())
+
+
+def voxelize(points, n_feat: int, batch_index: int, origin, voxel_size, grid_shape) -> dict:
+    """Voxelisation of raw points, the step the paper assumes upstream of its operators (Sec. II-A: a point cloud is
+    "partitioned into voxel grids" before the sparse tensor exists).  Plain definition, one point at a time.
+
+    ``points`` float32 ``[n, >= 3 + n_feat]`` rows ``(x, y, z, features...)``.  The cell of a point is
+    ``floor((p - origin) / voxel_size)`` per axis, taken in float32 exactly as written (subtract, divide, floor:
+    the decision is an integer, so both sides of a comparison must take it in the same precision); points whose
+    cell lies outside ``[0, grid_shape)`` are dropped.  Voxels are numbered in the order of their first point;
+    a voxel's features are the mean of its points' features (accumulated in float64).  Returns ``dict(coords int32
+    [m, 4] rows (batch_index, x, y, z), feats float64 [m, n_feat], counts int64 [m], voxel_of_point int64 [n] (-1 =
+    dropped))``.
+    """
+    pts = np.ascontiguousarray(points, dtype=np.float32)
+    o = np.asarray(origin, dtype=np.float32)
+    v = np.asarray(voxel_size, dtype=np.float32)
+    g = np.asarray(grid_shape, dtype=np.int64)
+    index_of = {}
+    coords, sums, counts = [], [], []
+    voxel_of_point = np.full(len(pts), -1, np.int64)
+    for i in range(len(pts)):
+        cell = []
+        inside = True
+        for a in range(3):
+            q = np.floor(np.float32(np.float32(pts[i, a] - o[a]) / v[a]))
+            if not (0 <= q < g[a]):
+                inside = False
+                break
+            cell.append(int(q))
+        if not inside:
+            continue
+        key = tuple(cell)
+        j = index_of.get(key)
+        if j is None:
+            j = len(coords)
+            index_of[key] = j
+            coords.append((batch_index,) + key)
+            sums.append(np.zeros(n_feat, np.float64))
+            counts.append(0)
+        sums[j] += pts[i, 3:3 + n_feat].astype(np.float64)
+        counts[j] += 1
+        voxel_of_point[i] = j
+    m = len(coords)
+    feats = np.array([s / c for s, c in zip(sums, counts)], np.float64).reshape(m, n_feat)
+    return dict(coords=np.array(coords, np.int32).reshape(m, 4), feats=feats, counts=np.array(counts, np.int64),
+                voxel_of_point=voxel_of_point)

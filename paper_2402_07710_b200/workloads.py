@@ -141,16 +141,12 @@ def indoor_surfaces(seed: int, target: int = 100_000, batch: int = 0) -> np.ndar
 LIDAR_GRID = (1408, 1600, 41)
 
 
-def lidar_sweep(seed: int, batch: int = 0) -> np.ndarray:
-    """One sweep of a synthetic 64-beam spinning LiDAR, voxelised (workload 3).
+LIDAR_ORIGIN = (-35.2, -40.0, -3.0)
+LIDAR_VOXEL = (0.05, 0.05, 0.1)
 
-    64 elevations uniform in [-25, +3] degrees x 2048 azimuth steps from a sensor
-    at the origin.  A ray stops at the ground plane z = -1.7 m or at the nearest
-    of 30 random boxes (edges 1.5-5 m, standing on the ground, centres at range
-    5-60 m and uniform bearing); hits beyond 70 m are dropped; range noise is
-    uniform +-2 cm.  Voxel size (0.05, 0.05, 0.1) m, grid 1408 x 1600 x 41 with
-    origin (-35.2, -40.0, -3.0) m so the sensor sits at the centre.
-    """
+
+def _lidar_hits(seed: int) -> np.ndarray:
+    """Hit points (float64 [m, 3], metres, sensor at the origin) of one synthetic sweep; see :func:`lidar_sweep`."""
     rng = np.random.default_rng(seed)
     el = np.deg2rad(np.linspace(-25.0, 3.0, 64))
     az = np.arange(2048) * (2.0 * np.pi / 2048)
@@ -173,12 +169,33 @@ def lidar_sweep(seed: int, batch: int = 0) -> np.ndarray:
         t = np.where(hit & (tn < t), tn, t)
     ok = t <= 70.0
     t = t[ok] + rng.uniform(-0.02, 0.02, int(ok.sum()))
-    p = d[ok] * t[:, None]
-    origin = np.array([-35.2, -40.0, -3.0])
-    vsize = np.array([0.05, 0.05, 0.1])
+    return d[ok] * t[:, None]
+
+
+def lidar_sweep(seed: int, batch: int = 0) -> np.ndarray:
+    """One sweep of a synthetic 64-beam spinning LiDAR, voxelised (workload 3).
+
+    64 elevations uniform in [-25, +3] degrees x 2048 azimuth steps from a sensor
+    at the origin.  A ray stops at the ground plane z = -1.7 m or at the nearest
+    of 30 random boxes (edges 1.5-5 m, standing on the ground, centres at range
+    5-60 m and uniform bearing); hits beyond 70 m are dropped; range noise is
+    uniform +-2 cm.  Voxel size (0.05, 0.05, 0.1) m, grid 1408 x 1600 x 41 with
+    origin (-35.2, -40.0, -3.0) m so the sensor sits at the centre.
+    """
+    p = _lidar_hits(seed)
+    origin = np.array(LIDAR_ORIGIN)
+    vsize = np.array(LIDAR_VOXEL)
     v = np.floor((p - origin) / vsize).astype(np.int64)
     keep = ((v >= 0) & (v < np.array(LIDAR_GRID))).all(axis=1)
     return _unique_rows(batch, v[keep])
+
+
+def lidar_points(seed: int, n_feat: int = 1) -> np.ndarray:
+    """The raw returns of the same sweep as float32 ``[m, 3 + n_feat]`` rows ``(x, y, z, features...)`` in beam
+    order, for the voxeliser: positions rounded to float32, features uniform in [0, 1) from a stream of their own."""
+    p = _lidar_hits(seed).astype(np.float32)
+    f = np.random.default_rng([seed, 0xFEA7]).random((len(p), n_feat), dtype=np.float32)
+    return np.ascontiguousarray(np.concatenate([p, f], axis=1))
 
 
 def lidar_batch(seeds=(0, 1, 2, 3)) -> np.ndarray:

@@ -392,3 +392,43 @@ def test_inverse_missing_parent_gives_zero_row_and_errors():
         oracle.build_inverse_kmap(np.array([[0, 1, 1, 1], [0, 1, 1, 1]], np.int32), coarse, 2, 2, 1)
     with pytest.raises(oracle.OracleError):
         oracle.build_inverse_kmap(fine, np.array([[0, -1, 0, 0]], np.int32), 2, 2, 1)
+
+
+# ----------------------------------------------------------------------------- voxelisation of raw points
+def test_voxelize_hand_example():
+    """Five points, voxel size 0.5 from origin (-1, -1, 0) on a 4 x 4 x 2 grid, worked by hand: two points share cell
+    (2, 2, 0) (their mean is the voxel's feature), one lies exactly on a cell boundary (it belongs to the upper
+    cell), one is outside the grid (dropped), cells are numbered by first appearance."""
+    pts = np.array([[0.10, 0.20, 0.30, 1.0, 10.0],     # cell (2, 2, 0)
+                    [-0.75, 0.90, 0.99, 2.0, 20.0],    # cell (0, 3, 1)
+                    [0.40, 0.49, 0.10, 3.0, 30.0],     # cell (2, 2, 0) again
+                    [0.00, -1.00, 0.50, 4.0, 40.0],    # exactly on boundaries: cell (2, 0, 1)
+                    [1.00, 0.00, 0.00, 5.0, 50.0]],    # x cell 4: outside
+                   np.float32)
+    r = oracle.voxelize(pts, 2, 7, (-1.0, -1.0, 0.0), (0.5, 0.5, 0.5), (4, 4, 2))
+    assert r["coords"].tolist() == [[7, 2, 2, 0], [7, 0, 3, 1], [7, 2, 0, 1]]
+    assert r["counts"].tolist() == [2, 1, 1]
+    assert np.allclose(r["feats"], [[2.0, 20.0], [2.0, 20.0], [4.0, 40.0]])
+    assert r["voxel_of_point"].tolist() == [0, 1, 0, 2, -1]
+
+
+def test_voxelize_agrees_with_the_workload_generator_and_library_routines():
+    """On the LiDAR returns the set of voxels equals what the workload generator builds with array operations
+    (unique rows of the floored positions, here in float32), counts sum to the points inside the grid, every
+    voxel's mean lies between its points' extremes, and a permutation of the points permutes the numbering only."""
+    pts = wl.lidar_points(5, n_feat=2)[:6000]
+    o, v, g = wl.LIDAR_ORIGIN, wl.LIDAR_VOXEL, wl.LIDAR_GRID
+    r = oracle.voxelize(pts, 2, 0, o, v, g)
+    cells = np.floor((pts[:, :3] - np.asarray(o, np.float32)) / np.asarray(v, np.float32)).astype(np.int64)
+    inside = ((cells >= 0) & (cells < np.asarray(g))).all(axis=1)
+    uniq, first, inv, cnt = np.unique(cells[inside], axis=0, return_index=True, return_inverse=True, return_counts=True)
+    order = np.argsort(first, kind="stable")                      # first appearance
+    assert np.array_equal(r["coords"][:, 1:], uniq[order])
+    assert np.array_equal(r["counts"], cnt[order]) and r["counts"].sum() == inside.sum()
+    sums = np.zeros((len(uniq), 2)); np.add.at(sums, inv.ravel(), pts[inside, 3:5].astype(np.float64))
+    assert np.allclose(r["feats"], (sums / cnt[:, None])[order], rtol=0, atol=1e-12)
+    perm = np.random.default_rng(1).permutation(len(pts))
+    r2 = oracle.voxelize(pts[perm], 2, 0, o, v, g)
+    a = {tuple(c): (f.round(12).tolist(), int(k)) for c, f, k in zip(r["coords"].tolist(), r["feats"], r["counts"])}
+    b = {tuple(c): (f.round(12).tolist(), int(k)) for c, f, k in zip(r2["coords"].tolist(), r2["feats"], r2["counts"])}
+    assert a.keys() == b.keys() and all(a[k][1] == b[k][1] and np.allclose(a[k][0], b[k][0], atol=1e-9) for k in a)
