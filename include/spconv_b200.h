@@ -278,6 +278,31 @@ int spconv_subm_offset_table_noalloc(const int32_t* coords, int64_t n, int kerne
                                      int32_t* nbr_out, void* cuda_stream);
 
 /*
+ * Voxelise raw points into the sparse tensor the operators take.  [Sec. II-A: the point cloud is "partitioned into
+ * voxel grids" and becomes an index list (m, x, y, z) plus a feature array; the paper assumes this step upstream]
+ *
+ *   points        device float32 [n][point_stride]: columns 0-2 are x, y, z (any unit), columns 3 .. 3 + n_feat - 1 the
+ *                 point's features; further columns are ignored.  Read only.
+ *   n_feat        >= 0 feature columns;  batch_index  0 .. 65534, written into column 0 of every output coordinate.
+ *   origin, voxel_size, grid_shape   HOST float[3], float[3] (> 0), int32[3] (1 .. 65535): the cell of a point is
+ *                 floor((p - origin) / voxel_size) per axis, evaluated in float32 exactly in that order; points whose
+ *                 cell is outside [0, grid_shape) are dropped.
+ *   coords_out    device int32 [capacity][4], 16-byte aligned: one row (batch_index, x, y, z) per occupied cell, in
+ *                 the order of the cells' first points (lowest point index first): the same on every run.
+ *   feats_out     device float32 [capacity][n_feat]: mean of the features of the cell's points (fp32 sums through
+ *                 atomic adds: the last bits may differ from run to run).  May be NULL when n_feat == 0.
+ *   counts_out    device int32 [capacity] or NULL: points per cell.
+ *   n_voxels_host HOST; receives the number of occupied cells.  If it exceeds `capacity` nothing is written to the
+ *                 outputs and the call returns SPCONV_ERR_TOO_LARGE (n_voxels_host still set, so the caller can retry).
+ * The call synchronises cuda_stream once (the caller has to learn the row count); the accumulation that follows is
+ * asynchronous.  coords_out can be passed to spconv_build_kmap as it is (rows are distinct and in range).
+ * Scratch memory comes from the device's stream-ordered pool.  Errors: INVALID_ARG, TOO_LARGE, TABLE_FULL, ALLOC, CUDA.
+ */
+int spconv_voxelize(const float* points, int64_t n, int point_stride, int n_feat, int batch_index, const float* origin /* host [3] */,
+                    const float* voxel_size /* host [3] */, const int32_t* grid_shape /* host [3] */, int32_t* coords_out,
+                    float* feats_out, int32_t* counts_out, int64_t capacity, int64_t* n_voxels_host /* host */, void* cuda_stream);
+
+/*
  * Diagnostics: copy the 16 status words that device kernels of this kernel map write to host memory `out16`
  * (synchronous copy).  Word 0: status bits (8 = a bounded wait of the tensor-core forward ran out); word 1: code of
  * the first wait that gave up (role << 24 | step, top bit set); word 2: its CTA + 1.  Cleared by the next build of a

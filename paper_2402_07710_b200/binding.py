@@ -23,7 +23,7 @@ DTYPE_BY_NAME = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloa
 EXPORTS = (
     "spconv_build_kmap", "spconv_build_inverse_kmap", "spconv_build_kmap_dense", "spconv_kmap_info", "spconv_kmap_destroy", "spconv_forward", "spconv_forward_algo",
     "spconv_last_device_status", "spconv_layer", "spconv_layer_host", "spconv_strerror", "spconv_subm_offset_table_noalloc",
-    "spconv_kmap_status_words", "spconv_test_hook",
+    "spconv_kmap_status_words", "spconv_test_hook", "spconv_voxelize",
 )
 HOOK_TABLE_SLOTS, HOOK_PIPE_WAIT_LIMIT_US = 1, 2
 NOALLOC_MAX_VOXELS = 131072
@@ -86,6 +86,9 @@ def load() -> ctypes.CDLL:
         lib.spconv_subm_offset_table_noalloc.argtypes = [vp, i64, i32, i32, vp, vp]
         lib.spconv_kmap_status_words.restype = i32
         lib.spconv_kmap_status_words.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+        lib.spconv_voxelize.restype = i32
+        lib.spconv_voxelize.argtypes = [vp, i64, i32, i32, i32, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float),
+                                        ctypes.POINTER(ctypes.c_int32), vp, vp, vp, i64, ctypes.POINTER(i64), vp]
         lib.spconv_test_hook.restype = i32
         lib.spconv_test_hook.argtypes = [i32, ctypes.c_longlong]
         lib.spconv_strerror.restype = ctypes.c_char_p
@@ -285,6 +288,31 @@ def spconv_layer(coords: torch.Tensor, feats: torch.Tensor, weights: torch.Tenso
 
 def spconv_last_device_status(kmap: Kmap, stream=None) -> int:
     return int(load().spconv_last_device_status(kmap._h, ctypes.c_void_p(_stream_ptr(stream))))
+
+
+def spconv_voxelize(points: torch.Tensor, n_feat: int, batch_index: int, origin, voxel_size, grid_shape, capacity: int | None = None,
+                    with_counts: bool = False, stream=None):
+    """Voxelise device points ``float32 [n, >= 3 + n_feat]``; returns ``(coords int32 [m, 4], feats float32 [m, n_feat])``
+    (and ``counts int32 [m]`` with ``with_counts``).  Output tensors are allocated here for ``capacity`` rows (default n)."""
+    if not (points.is_cuda and points.dtype == torch.float32 and points.dim() == 2 and points.is_contiguous()):
+        raise ValueError("points must be a contiguous CUDA float32 tensor [n, columns]")
+    n, stride = int(points.shape[0]), int(points.shape[1])
+    cap = n if capacity is None else int(capacity)
+    coords = torch.empty((max(cap, 1), 4), dtype=torch.int32, device=points.device)
+    feats = torch.empty((max(cap, 1), max(n_feat, 1)), dtype=torch.float32, device=points.device)
+    counts = torch.empty((max(cap, 1),), dtype=torch.int32, device=points.device) if with_counts else None
+    m = ctypes.c_int64(0)
+    st = load().spconv_voxelize(ctypes.c_void_p(points.data_ptr() if n else 0), n, stride, int(n_feat), int(batch_index),
+                                (ctypes.c_float * 3)(*[float(v) for v in origin]), (ctypes.c_float * 3)(*[float(v) for v in voxel_size]),
+                                (ctypes.c_int32 * 3)(*[int(v) for v in grid_shape]), ctypes.c_void_p(coords.data_ptr()),
+                                ctypes.c_void_p(feats.data_ptr() if n_feat else 0), ctypes.c_void_p(counts.data_ptr() if with_counts else 0),
+                                cap, ctypes.byref(m), ctypes.c_void_p(_stream_ptr(stream)))
+    if st != 0:
+        err = SpconvError(st, "spconv_voxelize")
+        err.n_voxels = int(m.value)
+        raise err
+    out = (coords[:m.value], feats[:m.value, :n_feat])
+    return out + (counts[:m.value],) if with_counts else out
 
 
 def spconv_kmap_status_words(kmap: Kmap) -> list:

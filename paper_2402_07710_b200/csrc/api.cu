@@ -260,6 +260,22 @@ int spconv_layer_host(const int32_t* coords_host, int64_t n, const void* feats_h
   return spconv_last_device_status(km, stream);
 }
 
+int spconv_voxelize(const float* points, int64_t n, int point_stride, int n_feat, int batch_index, const float* origin,
+                    const float* voxel_size, const int32_t* grid_shape, int32_t* coords_out, float* feats_out, int32_t* counts_out,
+                    int64_t capacity, int64_t* n_voxels_host, void* cuda_stream) {
+  if (n_voxels_host == nullptr) return SPCONV_ERR_INVALID_ARG;
+  *n_voxels_host = 0;
+  if (n < 0 || n > int64_t(1000000000) || n_feat < 0 || point_stride < 3 + n_feat || point_stride > 1024 || capacity < 0) return SPCONV_ERR_INVALID_ARG;
+  if (origin == nullptr || voxel_size == nullptr || grid_shape == nullptr) return SPCONV_ERR_INVALID_ARG;
+  if (batch_index < 0 || batch_index > kMaxCoord) return SPCONV_ERR_INVALID_ARG;
+  for (int a = 0; a < 3; ++a)
+    if (!(voxel_size[a] > 0.f) || grid_shape[a] < 1 || grid_shape[a] > kMaxCoord + 1) return SPCONV_ERR_INVALID_ARG;
+  if (n > 0 && (points == nullptr || coords_out == nullptr || (n_feat > 0 && feats_out == nullptr))) return SPCONV_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(coords_out) & 15u) return SPCONV_ERR_INVALID_ARG;
+  return voxelize_impl(points, n, point_stride, n_feat, batch_index, origin, voxel_size, grid_shape, coords_out, feats_out, counts_out,
+                       capacity, n_voxels_host, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int spconv_kmap_status_words(const spconv_kmap_t* km, uint32_t* out16) {
   if (km == nullptr || out16 == nullptr) return SPCONV_ERR_INVALID_ARG;
   if (km->d.status == nullptr) { std::memset(out16, 0, 64); return SPCONV_OK; }

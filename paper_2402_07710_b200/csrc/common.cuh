@@ -67,6 +67,10 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
 void destroy_kmap_impl(spconv_kmap* km);
 void set_kmap_test_table_slots(long long slots);          // test hook, see spconv_test_hook
 
+int voxelize_impl(const float* points, int64_t n, int point_stride, int n_feat, int batch_index, const float* origin,
+                  const float* voxel_size, const int32_t* grid_shape, int32_t* coords_out, float* feats_out, int32_t* counts_out,
+                  int64_t capacity, int64_t* n_voxels_host, cudaStream_t stream);
+
 // forward_simt.cu
 int forward_simt(const void* feats, const void* w, const spconv_kmap* km, void* out, int cin, int cout,
                  spconv_dtype_t dtype, cudaStream_t stream);

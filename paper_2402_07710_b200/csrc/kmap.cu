@@ -1746,6 +1746,133 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
 
 }  // namespace spconv
 
+
+// =============================================================================================
+// Voxelisation of raw points (see spconv_voxelize in the header): the step the paper assumes upstream of its
+// operators (Sec. II-A).  Built from the parts of the strided map: every point's cell is inserted into a hash table
+// of cells, the point with the lowest index owns the cell (atomicMin), cells are numbered in owner order -- the
+// order of their first point, the same on every run -- and then every point adds its features to its cell's row.
+namespace spconv {
+namespace {
+
+struct VoxGrid { float ox, oy, oz, vx, vy, vz; int gx, gy, gz, batch; };
+
+// One thread per point: the cell in float32 exactly as floor((p - origin) / voxel_size), points outside the grid dropped.
+__global__ void k_vox_cells(const float* __restrict__ points, int n, int stride_floats, const __grid_constant__ VoxGrid g,
+                            uint64_t* keys, int32_t* owner, uint32_t capmask, int32_t* __restrict__ point_slot, uint32_t* status) {
+  chain_begin();
+  const int i = blockIdx.x * kBlock + threadIdx.x;
+  if (i >= n) return;
+  const float* p = points + size_t(i) * stride_floats;
+  const float fx = floorf(__fdiv_rn(__fsub_rn(p[0], g.ox), g.vx)), fy = floorf(__fdiv_rn(__fsub_rn(p[1], g.oy), g.vy)),
+              fz = floorf(__fdiv_rn(__fsub_rn(p[2], g.oz), g.vz));
+  int slot = -1;
+  if (fx >= 0.f && fx < float(g.gx) && fy >= 0.f && fy < float(g.gy) && fz >= 0.f && fz < float(g.gz)) {
+    bool present;
+    slot = table_insert<1>(keys, capmask, pack_key(g.batch, int(fx), int(fy), int(fz)), &present);
+    if (slot < 0) atomicOr(status, kDevTableFull);
+    else atomicMin(owner + slot, i);
+  }
+  point_slot[i] = slot;
+}
+
+// One thread per (point, feature): the point's features are added to its voxel's row; thread 0 of a point counts it.
+__global__ void k_vox_accumulate(const float* __restrict__ points, int n, int stride_floats, int n_feat, const int32_t* __restrict__ point_slot,
+                                 const int32_t* __restrict__ slot_voxel, float* __restrict__ feats, int32_t* __restrict__ counts) {
+  chain_begin();
+  const int64_t e = int64_t(blockIdx.x) * kBlock + threadIdx.x;
+  const int cols = n_feat > 0 ? n_feat : 1;
+  const int64_t i = e / cols;
+  const int f = int(e - i * cols);
+  if (i >= n) return;
+  const int slot = point_slot[i];
+  if (slot < 0) return;
+  const int v = slot_voxel[slot];
+  if (n_feat > 0) atomicAdd(feats + size_t(v) * n_feat + f, points[size_t(i) * stride_floats + 3 + f]);
+  if (f == 0) atomicAdd(counts + v, 1);
+}
+
+__global__ void k_vox_normalize(float* __restrict__ feats, const int32_t* __restrict__ counts, int64_t m, int n_feat) {
+  chain_begin();
+  const int64_t e = int64_t(blockIdx.x) * kBlock + threadIdx.x;
+  if (e >= m * n_feat) return;
+  feats[e] = __fdiv_rn(feats[e], float(counts[e / n_feat]));
+}
+
+}  // namespace
+
+int voxelize_impl(const float* points, int64_t n, int point_stride, int n_feat, int batch_index, const float* origin,
+                  const float* voxel_size, const int32_t* grid_shape, int32_t* coords_out, float* feats_out, int32_t* counts_out,
+                  int64_t capacity, int64_t* n_voxels_host, cudaStream_t stream) {
+  *n_voxels_host = 0;
+  if (n == 0) return SPCONV_OK;
+  int device = 0;
+  SPCONV_CUDA_TRY(cudaGetDevice(&device));
+  keep_pool_cached(device);
+  const int nblk = int((n + kBlock - 1) / kBlock);
+  const uint32_t cap = pow2_at_least(uint64_t(2) * n);
+  const size_t totals_words = 8;
+  PinnedHost host;
+  host.count = totals_words + 2;
+  host.p = g_pinned.get(host.count);
+  if (!host.p) return SPCONV_ERR_ALLOC;
+  const size_t bytes = pad256(size_t(cap) * 8) + pad256(size_t(cap) * 4) * 2 + pad256(size_t(n) * 4) + pad256(size_t(nblk) * 4) +
+                       pad256(size_t(nblk) * 8) + pad256(totals_words * 8) + pad256(size_t(capacity > 0 ? capacity : 1) * 4) + 4096;
+  Scratch scratch;
+  scratch.stream = stream;
+  SPCONV_CUDA_TRY(cudaMallocAsync(&scratch.ptr, bytes, stream));
+  Arena sa{static_cast<char*>(scratch.ptr), bytes, 0};
+  uint64_t* keys = sa.take<uint64_t>(cap);
+  int32_t* owner = sa.take<int32_t>(cap);
+  int32_t* slot_voxel = sa.take<int32_t>(cap);
+  int32_t* point_slot = sa.take<int32_t>(n);
+  int32_t* cnt = sa.take<int32_t>(nblk);
+  int64_t* excl = sa.take<int64_t>(nblk);
+  int64_t* d_totals = sa.take<int64_t>(totals_words);
+  int32_t* own_counts = counts_out != nullptr ? counts_out : sa.take<int32_t>(size_t(capacity > 0 ? capacity : 1));
+  uint32_t* d_status = reinterpret_cast<uint32_t*>(d_totals + 2);
+  SPCONV_CUDA_TRY(cudaMemsetAsync(d_totals, 0, totals_words * 8, stream));
+  SPCONV_CUDA_TRY(cudaMemsetAsync(keys, 0xFF, size_t(cap) * 8, stream));
+  SPCONV_CUDA_TRY(cudaMemsetAsync(owner, 0x7F, size_t(cap) * 4, stream));
+  const VoxGrid g{origin[0], origin[1], origin[2], voxel_size[0], voxel_size[1], voxel_size[2], grid_shape[0], grid_shape[1], grid_shape[2], batch_index};
+  SPCONV_CUDA_TRY(launch_chained(k_vox_cells, dim3(nblk), dim3(kBlock), stream, points, int(n), point_stride, g, keys, owner, cap - 1, point_slot, d_status));
+  // owners = first points of their cells: counted per block, scanned, numbered (the strided map's kernels with one offset)
+  SPCONV_CUDA_TRY(launch_chained(k_owner_count, dim3(nblk, 1), dim3(kBlock), stream, static_cast<const int32_t*>(point_slot),
+                                 static_cast<const int32_t*>(owner), int(n), cnt));
+  SPCONV_CUDA_TRY(launch_chained(k_scan_counts, dim3(1), dim3(1024), stream, static_cast<const int32_t*>(cnt), int64_t(nblk), excl, nblk, 1,
+                                 static_cast<int64_t*>(nullptr), d_totals + 0, static_cast<int8_t*>(nullptr)));
+  volatile int64_t* ready = host.p + totals_words;
+  *ready = 0;
+  host.writer = stream;
+  host.write_pending = true;
+  SPCONV_CUDA_TRY(launch_chained(k_report_totals, dim3(1), dim3(64), stream, static_cast<const int64_t*>(d_totals), int(totals_words), host.p));
+  SPCONV_CUDA_TRY(cudaStreamSynchronize(stream));   // one wait: the caller needs the number of voxels
+  host.write_pending = false;
+  if (*ready != 1) return SPCONV_ERR_CUDA;
+  if (uint32_t(host.p[2]) & kDevTableFull) return SPCONV_ERR_TABLE_FULL;
+  const int64_t m = host.p[0];
+  *n_voxels_host = m;
+  if (m > capacity) return SPCONV_ERR_TOO_LARGE;
+  if (m == 0) return SPCONV_OK;
+  SPCONV_CUDA_TRY(launch_chained(k_owner_assign, dim3(nblk, 1), dim3(kBlock), stream, static_cast<const int32_t*>(point_slot),
+                                 static_cast<const int32_t*>(owner), static_cast<const uint64_t*>(keys), int(n),
+                                 static_cast<const int64_t*>(excl), slot_voxel, reinterpret_cast<int4*>(coords_out)));
+  if (n_feat > 0) SPCONV_CUDA_TRY(cudaMemsetAsync(feats_out, 0, size_t(m) * n_feat * 4, stream));
+  SPCONV_CUDA_TRY(cudaMemsetAsync(own_counts, 0, size_t(m) * 4, stream));
+  const int cols = n_feat > 0 ? n_feat : 1;
+  const int64_t acc_threads = n * cols;
+  SPCONV_CUDA_TRY(launch_chained(k_vox_accumulate, dim3(unsigned((acc_threads + kBlock - 1) / kBlock)), dim3(kBlock), stream, points, int(n),
+                                 point_stride, n_feat, static_cast<const int32_t*>(point_slot), static_cast<const int32_t*>(slot_voxel), feats_out,
+                                 own_counts));
+  if (n_feat > 0)
+    SPCONV_CUDA_TRY(launch_chained(k_vox_normalize, dim3(unsigned((m * n_feat + kBlock - 1) / kBlock)), dim3(kBlock), stream, feats_out,
+                                   static_cast<const int32_t*>(own_counts), m, n_feat));
+  SPCONV_CUDA_TRY(cudaGetLastError());
+  return SPCONV_OK;
+}
+
+}  // namespace spconv
+
 // =============================================================================================
 // Offset table without any allocation (see spconv_subm_offset_table_noalloc in the header).
 //
