@@ -67,7 +67,9 @@ typedef enum {
 typedef enum {
   SPCONV_ALGO_AUTO = 0,
   SPCONV_ALGO_SIMT = 1,    /* fp32 FMA on CUDA cores (any dtype; the only exact-fp32 path) */
-  SPCONV_ALGO_TCGEN05 = 2  /* implicit GEMM on 5th-gen tensor cores, fp32 accumulators in TMEM */
+  SPCONV_ALGO_TCGEN05 = 2, /* implicit GEMM on 5th-gen tensor cores, fp32 accumulators in TMEM; a pipeline step takes as
+                              many offsets of a tile as the shape allows (four for 16/32 channels in, two for 64 -> <=64) */
+  SPCONV_ALGO_TCGEN05_SINGLE = 3 /* the same kernel with one offset per step (fixed grouping of one): for comparison */
 } spconv_algo_t;
 
 typedef struct {
@@ -113,6 +115,22 @@ typedef struct {
  */
 int spconv_build_kmap(const int32_t* coords, int64_t n, int stride, int dilation, int kernel_size,
                       int submanifold, void* cuda_stream, spconv_kmap_t** kmap_out);
+
+/*
+ * spconv_build_kmap with the order of the tensor-core forward's row tiles chosen by the caller.  [Related work of
+ * Sec. II-C: how (input, output) pairs are grouped into matrix products decides the padding they carry]
+ *   SPCONV_ROWS_BY_OFFSET_SET  (what spconv_build_kmap does) rows sorted by the set of offsets through which they have
+ *                              an input, so that a 128-row tile needs few offsets and its (tile, offset) blocks are
+ *                              well filled; costs a sort per build.
+ *   SPCONV_ROWS_AS_GIVEN       tile t holds output rows 128 t .. 128 t + 127: no sort (a shorter build), more and
+ *                              emptier blocks (a slower forward), input rows of a tile close together when the caller's
+ *                              row order is spatially coherent (e.g. Morton-sorted coordinates).
+ * The kernel map itself (offset table, pairs, output coordinates) is the same for both; only the tile plan differs,
+ * and with it the speed, never the result, of the tensor-core forward.
+ */
+typedef enum { SPCONV_ROWS_BY_OFFSET_SET = 0, SPCONV_ROWS_AS_GIVEN = 1 } spconv_row_order_t;
+int spconv_build_kmap_ordered(const int32_t* coords, int64_t n, int stride, int dilation, int kernel_size, int submanifold,
+                              int row_order, void* cuda_stream, spconv_kmap_t** kmap_out);
 
 /*
  * Build the kernel map of an inverse (transposed) convolution, the up-sampling counterpart of a strided layer.

@@ -16,12 +16,13 @@ _DIR = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_DIR, "libspconv_b200.so")
 
 F32, F16, BF16 = 0, 1, 2
-ALGO = {"auto": 0, "simt": 1, "tcgen05": 2}
+ALGO = {"auto": 0, "simt": 1, "tcgen05": 2, "tcgen05_single": 3}
+ROWS_BY_OFFSET_SET, ROWS_AS_GIVEN = 0, 1
 _TORCH_DTYPE = {torch.float32: F32, torch.float16: F16, torch.bfloat16: BF16}
 DTYPE_BY_NAME = {"f32": torch.float32, "f16": torch.float16, "bf16": torch.bfloat16}
 
 EXPORTS = (
-    "spconv_build_kmap", "spconv_build_inverse_kmap", "spconv_build_kmap_dense", "spconv_kmap_info", "spconv_kmap_destroy", "spconv_forward", "spconv_forward_algo",
+    "spconv_build_kmap", "spconv_build_kmap_ordered", "spconv_build_inverse_kmap", "spconv_build_kmap_dense", "spconv_kmap_info", "spconv_kmap_destroy", "spconv_forward", "spconv_forward_algo",
     "spconv_last_device_status", "spconv_layer", "spconv_layer_host", "spconv_strerror", "spconv_subm_offset_table_noalloc",
     "spconv_kmap_status_words", "spconv_test_hook", "spconv_voxelize",
 )
@@ -63,6 +64,8 @@ def load() -> ctypes.CDLL:
         vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
         lib.spconv_build_kmap.restype = i32
         lib.spconv_build_kmap.argtypes = [vp, i64, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
+        lib.spconv_build_kmap_ordered.restype = i32
+        lib.spconv_build_kmap_ordered.argtypes = [vp, i64, i32, i32, i32, i32, i32, vp, ctypes.POINTER(vp)]
         lib.spconv_build_inverse_kmap.restype = i32
         lib.spconv_build_inverse_kmap.argtypes = [vp, i64, vp, i64, i32, i32, i32, vp, ctypes.POINTER(vp)]
         lib.spconv_build_kmap_dense.restype = i32
@@ -185,12 +188,20 @@ class Kmap:
 
 
 def spconv_build_kmap(coords: torch.Tensor, stride: int = 1, dilation: int = 1, kernel_size: int = 3,
-                      submanifold: bool = True, stream=None) -> Kmap:
-    """Build the kernel map of one layer from device coordinates ``int32 [n, 4]`` rows (b, x, y, z)."""
+                      submanifold: bool = True, stream=None, row_order: int | None = None) -> Kmap:
+    """Build the kernel map of one layer from device coordinates ``int32 [n, 4]`` rows (b, x, y, z).
+    ``row_order`` (``ROWS_BY_OFFSET_SET`` / ``ROWS_AS_GIVEN``) goes through ``spconv_build_kmap_ordered``."""
     if not (coords.is_cuda and coords.dtype == torch.int32 and coords.dim() == 2 and coords.shape[1] == 4
             and coords.is_contiguous()):
         raise ValueError("coords must be a contiguous CUDA int32 tensor of shape [n, 4]")
     h = ctypes.c_void_p(None)
+    if row_order is not None:
+        st = load().spconv_build_kmap_ordered(ctypes.c_void_p(coords.data_ptr() if coords.numel() else 0), coords.shape[0],
+                                              int(stride), int(dilation), int(kernel_size), int(bool(submanifold)), int(row_order),
+                                              ctypes.c_void_p(_stream_ptr(stream)), ctypes.byref(h))
+        if st != 0:
+            raise SpconvError(st, "spconv_build_kmap_ordered")
+        return Kmap(h.value)
     st = load().spconv_build_kmap(ctypes.c_void_p(coords.data_ptr() if coords.numel() else 0), coords.shape[0],
                                   int(stride), int(dilation), int(kernel_size), int(bool(submanifold)),
                                   ctypes.c_void_p(_stream_ptr(stream)), ctypes.byref(h))

@@ -30,7 +30,8 @@ const char* spconv_strerror(int status) {
 namespace {
 // spconv_build_kmap with build_kmap_impl's before_wait hook (used by spconv_layer).
 int spconv_build_kmap_hooked(const int32_t* coords, int64_t n, int stride, int dilation, int kernel_size, int submanifold,
-                             void* cuda_stream, spconv_kmap_t** kmap_out, const std::function<int(spconv_kmap*)>* before_wait) {
+                             void* cuda_stream, spconv_kmap_t** kmap_out, const std::function<int(spconv_kmap*)>* before_wait,
+                             int rows_as_given = 0) {
   if (kmap_out == nullptr) return SPCONV_ERR_INVALID_ARG;
   *kmap_out = nullptr;
   if (n < 0 || stride < 1 || dilation < 1 || kernel_size < 1) return SPCONV_ERR_INVALID_ARG;
@@ -41,13 +42,24 @@ int spconv_build_kmap_hooked(const int32_t* coords, int64_t n, int stride, int d
   if (submanifold && (stride != 1 || kernel_size % 2 == 0)) return SPCONV_ERR_INVALID_ARG;
   const int64_t kvol = int64_t(kernel_size) * kernel_size * kernel_size;
   if (n * kvol > int64_t(2000000000)) return SPCONV_ERR_TOO_LARGE;
-  return build_kmap_impl(coords, n, stride, dilation, kernel_size, submanifold, static_cast<cudaStream_t>(cuda_stream), kmap_out, before_wait);
+  return build_kmap_impl(coords, n, stride, dilation, kernel_size, submanifold, static_cast<cudaStream_t>(cuda_stream), kmap_out, before_wait,
+                         nullptr, 0, nullptr, rows_as_given);
 }
 }  // namespace
 
 int spconv_build_kmap(const int32_t* coords, int64_t n, int stride, int dilation, int kernel_size, int submanifold,
                       void* cuda_stream, spconv_kmap_t** kmap_out) {
   return spconv_build_kmap_hooked(coords, n, stride, dilation, kernel_size, submanifold, cuda_stream, kmap_out, nullptr);
+}
+
+int spconv_build_kmap_ordered(const int32_t* coords, int64_t n, int stride, int dilation, int kernel_size, int submanifold,
+                              int row_order, void* cuda_stream, spconv_kmap_t** kmap_out) {
+  if (row_order != SPCONV_ROWS_BY_OFFSET_SET && row_order != SPCONV_ROWS_AS_GIVEN) {
+    if (kmap_out != nullptr) *kmap_out = nullptr;
+    return SPCONV_ERR_INVALID_ARG;
+  }
+  return spconv_build_kmap_hooked(coords, n, stride, dilation, kernel_size, submanifold, cuda_stream, kmap_out, nullptr,
+                                  row_order == SPCONV_ROWS_AS_GIVEN ? 1 : 0);
 }
 
 int spconv_build_inverse_kmap(const int32_t* fine_coords, int64_t n_fine, const int32_t* coarse_coords, int64_t n_coarse,
@@ -127,6 +139,8 @@ int forward_checked(const void* feats, const void* weights, const spconv_kmap_t*
       return forward_simt(feats, weights, km, out, cin, cout, dtype, stream);
     case SPCONV_ALGO_TCGEN05:
       return forward_tc(feats, weights, km, out, cin, cout, dtype, stream, strict_order);
+    case SPCONV_ALGO_TCGEN05_SINGLE:
+      return forward_tc(feats, weights, km, out, cin, cout, dtype, stream, strict_order, true);
   }
   return SPCONV_ERR_INVALID_ARG;
 }

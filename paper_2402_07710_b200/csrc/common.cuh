@@ -61,7 +61,7 @@ namespace spconv {
 // (rows of the input features), fine_coords [n_fine][4] the output rows, and submanifold must be 0.
 int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, int kernel, int submanifold,
                     cudaStream_t stream, spconv_kmap** out, const std::function<int(spconv_kmap*)>* before_wait = nullptr,
-                    const int32_t* fine_coords = nullptr, int64_t n_fine = 0, const int* dense_grid = nullptr);
+                    const int32_t* fine_coords = nullptr, int64_t n_fine = 0, const int* dense_grid = nullptr, int rows_as_given = 0);
 // dense_grid (optional, host int[4] = B, X, Y, Z): the location table is a dense array over that grid instead of the
 // hash table (submanifold maps with kernel size 1 or 3 only; the caller checks the shape and its size).
 void destroy_kmap_impl(spconv_kmap* km);
@@ -81,8 +81,9 @@ void set_forward_tc_timeline(unsigned long long* buf);
 void set_forward_tc_test_wait_limit_us(long long us);     // test hook, see spconv_test_hook
 // strict_order: the kernel map may still be under construction by work that precedes the launch in the stream
 // (the launch comes from build_kmap_impl's before_wait), so the kernel must not read it ahead of that work.
+// one_offset_per_step: never take several offsets of a tile in one pipeline step (SPCONV_ALGO_TCGEN05_SINGLE).
 int forward_tc(const void* feats, const void* w, const spconv_kmap* km, void* out, int cin, int cout,
-               spconv_dtype_t dtype, cudaStream_t stream, bool strict_order = false);
+               spconv_dtype_t dtype, cudaStream_t stream, bool strict_order = false, bool one_offset_per_step = false);
 
 inline int dtype_size(spconv_dtype_t t) { return t == SPCONV_F32 ? 4 : 2; }
 

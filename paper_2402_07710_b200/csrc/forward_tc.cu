@@ -1161,7 +1161,16 @@ int launch(const void* feats, const void* w, const spconv_kmap* km, void* out, s
 
 template <int CIN>
 int dispatch_cout(const void* feats, const void* w, const spconv_kmap* km, void* out, int cout, spconv_dtype_t dtype,
-                  cudaStream_t stream, bool strict_order) {
+                  cudaStream_t stream, bool strict_order, bool single) {
+  if (single) {
+    switch (cout) {
+      case 16: return launch<CIN, 16, false>(feats, w, km, out, dtype, stream, strict_order);
+      case 32: return launch<CIN, 32, false>(feats, w, km, out, dtype, stream, strict_order);
+      case 64: return launch<CIN, 64, false>(feats, w, km, out, dtype, stream, strict_order);
+      case 128: return launch<CIN, 128, false>(feats, w, km, out, dtype, stream, strict_order);
+    }
+    return SPCONV_ERR_INVALID_ARG;
+  }
   switch (cout) {
     case 16: return (grouped_shape(CIN, 16) && km->kvol <= 32) ? launch<CIN, 16, grouped_shape(CIN, 16)>(feats, w, km, out, dtype, stream, strict_order)
                                                                   : launch<CIN, 16, false>(feats, w, km, out, dtype, stream, strict_order);
@@ -1190,14 +1199,14 @@ bool forward_tc_supported(int cin, int cout, spconv_dtype_t dtype) {
 }
 
 int forward_tc(const void* feats, const void* w, const spconv_kmap* km, void* out, int cin, int cout,
-               spconv_dtype_t dtype, cudaStream_t stream, bool strict_order) {
+               spconv_dtype_t dtype, cudaStream_t stream, bool strict_order, bool one_offset_per_step) {
   if (!forward_tc_supported(cin, cout, dtype) || km->kvol > 128) return SPCONV_ERR_INVALID_ARG;
   if (km->n_out == 0) return SPCONV_OK;
   switch (cin) {
-    case 16: return dispatch_cout<16>(feats, w, km, out, cout, dtype, stream, strict_order);
-    case 32: return dispatch_cout<32>(feats, w, km, out, cout, dtype, stream, strict_order);
-    case 64: return dispatch_cout<64>(feats, w, km, out, cout, dtype, stream, strict_order);
-    case 128: return dispatch_cout<128>(feats, w, km, out, cout, dtype, stream, strict_order);
+    case 16: return dispatch_cout<16>(feats, w, km, out, cout, dtype, stream, strict_order, one_offset_per_step);
+    case 32: return dispatch_cout<32>(feats, w, km, out, cout, dtype, stream, strict_order, one_offset_per_step);
+    case 64: return dispatch_cout<64>(feats, w, km, out, cout, dtype, stream, strict_order, one_offset_per_step);
+    case 128: return dispatch_cout<128>(feats, w, km, out, cout, dtype, stream, strict_order, one_offset_per_step);
   }
   return SPCONV_ERR_INVALID_ARG;
 }

@@ -1319,7 +1319,7 @@ struct TimelineDump {
 
 int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, int kernel, int submanifold,
                     cudaStream_t stream, spconv_kmap** out, const std::function<int(spconv_kmap*)>* before_wait,
-                    const int32_t* fine_coords, int64_t n_fine, const int* dense_grid) {
+                    const int32_t* fine_coords, int64_t n_fine, const int* dense_grid, int rows_as_given) {
   [[maybe_unused]] StageTimer stages(stream);
 #ifdef SPCONV_KMAP_TIMELINE
   TimelineDump timeline_dump{stream};
@@ -1382,7 +1382,9 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     n_out_max = std::min<int64_t>(n * int64_t(cpa) * cpa * cpa, int64_t(2000000000));
     cap2 = pow2_at_least(uint64_t(2) * n_out_max);
   }
-  const bool plan_sorted = kvol <= 32;   // the tile plan sorts rows by their offset set when it fits one 32-bit key
+  // The tile plan sorts rows by their offset set when it fits one 32-bit key, unless the caller asked for tiles of
+  // consecutive rows (SPCONV_ROWS_AS_GIVEN: no sort, more (tile, offset) blocks).
+  const bool plan_sorted = kvol <= 32 && !rows_as_given;
   // The radix sort takes 8 bits per pass; the three passes over the 24 most significant key bits (the rarest
   // offsets) already bring the block count within a few per cent of the full sort's.
   const int sort_begin_bit = kvol > 24 ? kvol - 24 : 0;
