@@ -502,6 +502,99 @@ def run_survey(args):
     print(json.dumps({"survey": rows, "peaks": peaks}))
 
 
+def run_options(args):
+    """The measured options of the path (not the bench line), one JSON line: row order of the tile plan x offsets per
+    pipeline step of the tensor-core forward; hash table against dense-array location table; the voxeliser."""
+    import numpy as np
+    import torch
+
+    from paper_2402_07710_b200 import binding
+
+    torch.cuda.set_device(0)
+    stream = torch.cuda.current_stream()
+
+    def build_time(fn, reps=20):          # median of event-timed calls through the Python binding, microseconds
+        ts = []
+        for i in range(reps + 3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            r = fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b) * 1e3)
+            if hasattr(r, "close"):
+                r.close()
+        return statistics.median(ts)
+
+    def graph_time(fn, launches=20):      # microseconds per launch, CUDA-graph replay on L2-warm arrays
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            for _ in range(launches):
+                fn()
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(5):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            g.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) / launches * 1e3)
+        return statistics.median(ts)
+
+    def z_order(c):                        # rows sorted along a Z-order curve (batch-major)
+        def spread(v):
+            v = v.astype(np.uint64) & np.uint64(0x1fffff)
+            v = (v | (v << np.uint64(32))) & np.uint64(0x1f00000000ffff)
+            v = (v | (v << np.uint64(16))) & np.uint64(0x1f0000ff0000ff)
+            v = (v | (v << np.uint64(8))) & np.uint64(0x100f00f00f00f00f)
+            v = (v | (v << np.uint64(4))) & np.uint64(0x10c30c30c30c30c3)
+            v = (v | (v << np.uint64(2))) & np.uint64(0x1249249249249249)
+            return v
+        key = (c[:, 0].astype(np.uint64) << np.uint64(60)) | (spread(c[:, 1]) << np.uint64(2)) | (spread(c[:, 2]) << np.uint64(1)) | spread(c[:, 3])
+        return np.ascontiguousarray(c[np.argsort(key, kind="stable")])
+
+    c3, c2 = wl.config(3)["coords"], wl.config(2)["coords"]
+    cases = [("config 3, rows as generated (scan order)", c3, 3, 1, True, 64, 64),
+             ("config 3, rows shuffled", wl.shuffle_rows(c3, seed=1), 3, 1, True, 64, 64),
+             ("config 3, rows in Z-order", z_order(c3), 3, 1, True, 64, 64),
+             ("config 2, rows as generated", c2, 3, 1, True, 32, 32),
+             ("config 2, rows in Z-order", z_order(c2), 3, 1, True, 32, 32),
+             ("config 4 L0 (K3 s2)", c3, 3, 2, False, 64, 128),
+             ("config 4 L1 (K2 s2)", c3, 2, 2, False, 64, 64)]
+    row_options = []
+    for name, coords, K, s, subm, cin, cout in cases:
+        t = torch.from_numpy(np.ascontiguousarray(coords)).cuda()
+        for order, oname in ((binding.ROWS_BY_OFFSET_SET, "by offset set"), (binding.ROWS_AS_GIVEN, "as given")):
+            km = binding.spconv_build_kmap(t, s, 1, K, subm, row_order=order)
+            tb = build_time(lambda: binding.spconv_build_kmap(t, s, 1, K, subm, row_order=order))
+            x = torch.randn(km.n_in, cin, device="cuda").bfloat16()
+            w = torch.randn(K ** 3, cin, cout, device="cuda").bfloat16()
+            out = torch.empty(km.n_out, cout, device="cuda", dtype=torch.bfloat16)
+            tg = graph_time(lambda: binding.spconv_forward(x, w, km, algo="tcgen05", out=out))
+            ts = graph_time(lambda: binding.spconv_forward(x, w, km, algo="tcgen05_single", out=out))
+            row_options.append(dict(case=name, rows=km.n_out, order=oname, tile_blocks=km.tile_blocks, kmap_build_us=tb,
+                                    forward_us_offsets_grouped=tg, forward_us_one_offset_per_step=ts))
+            km.close()
+    tables = []
+    c1 = torch.from_numpy(wl.config(1)["coords"]).cuda()
+    blob = torch.from_numpy(wl.shuffle_rows(wl.random_blob(60000, 50, seed=3, batches=2), seed=1)).cuda()
+    for name, c, grid in (("config 1 (%d voxels), grid 1 x 64^3" % len(c1), c1, (1, 64, 64, 64)),
+                          ("blob (%d voxels), grid 2 x 128^3" % len(blob), blob, (2, 128, 128, 128))):
+        tables.append(dict(input=name, hash_table_build_us=build_time(lambda: binding.spconv_build_kmap(c, 1, 1, 3, True)),
+                           dense_array_build_us=build_time(lambda: binding.spconv_build_kmap_dense(c, grid, 1, 3))))
+    pts = torch.from_numpy(wl.lidar_points(0, n_feat=4)).cuda()
+    vc, _ = binding.spconv_voxelize(pts, 4, 0, wl.LIDAR_ORIGIN, wl.LIDAR_VOXEL, wl.LIDAR_GRID)
+    vox = dict(points=len(pts), n_feat=4, voxels=len(vc),
+               us=build_time(lambda: binding.spconv_voxelize(pts, 4, 0, wl.LIDAR_ORIGIN, wl.LIDAR_VOXEL, wl.LIDAR_GRID)[0]))
+    print(json.dumps({"row_options": row_options, "location_table": tables, "voxelize": vox}))
+
+
 def respawn_under_torchrun(args):
     """`python bench.py --gpus N` with N > 1 and no launcher around it: start the N ranks here (one per GPU, NCCL
     rendezvous on 127.0.0.1) and pass their output through."""
@@ -524,11 +617,15 @@ def main():
     ap.add_argument("--only", choices=("forward", "kmap"), default=None,
                     help="run three launches of one stage and exit (for profiler captures)")
     ap.add_argument("--survey", action="store_true", help="per-layer table over all five workloads (one JSON line)")
+    ap.add_argument("--options", action="store_true",
+                    help="row order x offsets per step, hash table vs dense array, voxeliser (one JSON line)")
     args = ap.parse_args()
-    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.survey and not args.only:
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and not args.survey and not args.options and not args.only:
         sys.exit(respawn_under_torchrun(args))
     if args.survey:
         run_survey(args)
+    elif args.options:
+        run_options(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

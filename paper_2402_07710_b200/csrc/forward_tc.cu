@@ -47,7 +47,10 @@ constexpr int kMaxPipes = 2;                     // independent gather -> MMA pi
 constexpr int kGroupWarps = 8;                   // producer warps of one pipeline (they share a step's rows)
 constexpr int kGroupThreads = 32 * kGroupWarps;
 constexpr int kMaxAStages = 12;                  // most stages a CTA's rings hold in all
-constexpr int kInStageMin = 3;                   // a stage carries its W_k where at least this many stages per pipeline fit
+#ifndef SPCONV_X_INSTAGE_MIN
+#define SPCONV_X_INSTAGE_MIN 3
+#endif
+constexpr int kInStageMin = SPCONV_X_INSTAGE_MIN;                   // a stage carries its W_k where at least this many stages per pipeline fit
 constexpr int kGroupMaxCin = 64;                 // widest input rows that take several offsets per step
 // Shapes that take several offsets per step: short rows always; 128-byte rows (two offsets) only where two such stages per pipeline fit.
 constexpr bool grouped_shape(int cin, int cout) { return cin <= kGroupMaxCin && (cin < 64 || cout <= 64); }
