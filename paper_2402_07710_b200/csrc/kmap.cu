@@ -293,18 +293,28 @@ k_probe_rows(const int4* __restrict__ qcoords, int nq, int dil, int stride, cons
 #pragma unroll
     for (int k = 0; k < KV; ++k) s_v[k][tid] = (MODE == 0 && k == (r * K + r) * K + r && live) ? j : got[k];
   } else {
-    uint32_t word[KV];
+    // The filter keeps the 64 z-positions of a line (b, x, y) in two neighbouring words, so one 8-byte load serves the
+    // K offsets of a line: K x K loads per row instead of K^3.
+    uint2 line[K * K];
+#pragma unroll
+    for (int l = 0; l < K * K; ++l) {
+      int x, y, z;
+      // (a line is read if any of its K offsets has a position at all; x and y are the same for all of them)
+      bool any = false;
+#pragma unroll
+      for (int cc = 0; cc < K; ++cc) { int x2, y2, z2; if (target(l * K + cc, x2, y2, z2)) { any = true; x = x2; y = y2; z = z2; } }
+      line[l] = make_uint2(0xFFFFFFFFu, 0xFFFFFFFFu);
+      if (any) line[l] = occ != nullptr ? __ldg(reinterpret_cast<const uint2*>(occ + (occ_word(c.x, x, y, z) & ~1u))) : make_uint2(0u, 0u);
+    }
 #pragma unroll
     for (int k = 0; k < KV; ++k) {
       int x, y, z;
       const bool valid = target(k, x, y, z);
-      word[k] = 0xFFFFFFFFu;
-      if (valid) word[k] = occ != nullptr ? __ldg(occ + occ_word(c.x, x, y, z)) : 0u;
-      word[k] = (word[k] >> (z & 31)) & 1u;   // 1: ruled out
+      const uint32_t w = (z & 32) ? line[k / K].y : line[k / K].x;
+      const uint32_t out = valid ? ((w >> (z & 31)) & 1u) : 1u;   // 1: ruled out
+      cand |= (out ^ 1u) << k;
       s_v[k][tid] = (MODE == 0 && k == (r * K + r) * K + r && live) ? j : -1;
     }
-#pragma unroll
-    for (int k = 0; k < KV; ++k) cand |= (word[k] ^ 1u) << k;
   }
   // 2. the candidates' table lookups, four at a time
   while (cand != 0u) {
