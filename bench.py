@@ -47,10 +47,11 @@ REFERENCE_SAMPLE_VOXELS = 10**9   # the oracle finishes the whole sweep in a fra
 FORWARD_DRAM_TRAFFIC_BYTES = 15_232_512
 FORWARD_DRAM_TRAFFIC_SOURCE = ("one profiler capture of k_forward_tc<64,64> on sweep 0 (DRAM bytes read + written per launch, "
                                "caches flushed before the launch); recorded, not measured in this run")
-# Our kernels launched per step: k_insert, k_probe_rows (every offset of a row per thread), k_subm_emit (on a second
+# Our kernels launched per step: k_fill_regions (table, filter, totals), k_insert, k_probe_rows (every offset of a row
+# per thread), k_subm_emit (on a second
 # stream), k_sort_rows_coop (row keys + radix sort, one cooperative launch), k_tile_plan_rows (its last block also
 # orders the tiles and reports to the host) for the kernel map, + k_forward_tc.
-OUR_LAUNCHES_PER_STEP = 6
+OUR_LAUNCHES_PER_STEP = 7
 ROTATION = 8   # sweeps a rank rotates over (about 45 MB of arrays each)
 
 

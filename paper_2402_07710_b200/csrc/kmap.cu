@@ -46,6 +46,16 @@ __device__ __forceinline__ void tl_stamp(int slot) {
 #define SPCONV_TL(slot)
 #define SPCONV_TL_RAW(slot, t)
 #endif
+// The fills a build starts with (location table and filter to all ones, totals to zero, the strided path's second
+// table and owner words), as one kernel in the chain instead of separate memset nodes, which programmatic dependent
+// launch cannot chain: between two builds of a sequence the launch latencies of those nodes were dead time.
+struct FillRegions {
+  uint4* ptr[4];
+  unsigned long long count16[4];   // 16-byte words
+  uint32_t value[4];
+};
+__global__ void __launch_bounds__(256) k_fill_regions(const __grid_constant__ FillRegions regions);
+
 template <class... Params, class... Args>
 cudaError_t launch_chained(void (*kernel)(Params...), dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
   cudaLaunchConfig_t config = {};
@@ -1165,6 +1175,16 @@ SideStream* side_stream_for(int device) {
   return &side;
 }
 
+__global__ void __launch_bounds__(256) k_fill_regions(const __grid_constant__ FillRegions regions) {
+  chain_begin();
+  const size_t stride = size_t(gridDim.x) * blockDim.x, first = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const uint4 v = make_uint4(regions.value[r], regions.value[r], regions.value[r], regions.value[r]);
+    for (size_t i = first; i < regions.count16[r]; i += stride) regions.ptr[r][i] = v;
+  }
+}
+
 uint32_t pow2_at_least(uint64_t v) {
   uint64_t c = 64;
   while (c < v) c <<= 1;
@@ -1601,8 +1621,19 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     return SPCONV_OK;
   };
 
-  SPCONV_CUDA_TRY(cudaMemsetAsync(d_totals, 0, (totals_words + 16) * sizeof(int64_t), stream));
-  SPCONV_CUDA_TRY(cudaMemsetAsync(table1, 0xFF, table_fill_bytes, stream));
+  {  // (every region starts on a 256-byte boundary of the arena and is followed by padding up to the next one, so
+     // rounding a size up to 16 bytes stays inside its own padding)
+    FillRegions fr = {};
+    fr.ptr[0] = reinterpret_cast<uint4*>(d_totals); fr.count16[0] = ((totals_words + 16) * sizeof(int64_t) + 15) / 16; fr.value[0] = 0u;
+    fr.ptr[1] = reinterpret_cast<uint4*>(table1); fr.count16[1] = (table_fill_bytes + 15) / 16; fr.value[1] = 0xFFFFFFFFu;
+    if (!known_outputs) {
+      fr.ptr[2] = reinterpret_cast<uint4*>(keys2); fr.count16[2] = size_t(cap2) * 8 / 16; fr.value[2] = 0xFFFFFFFFu;
+      fr.ptr[3] = reinterpret_cast<uint4*>(owner_cid); fr.count16[3] = size_t(cap2) * 4 / 16; fr.value[3] = 0x7F7F7F7Fu;
+    }
+    const size_t words = fr.count16[0] + fr.count16[1] + fr.count16[2] + fr.count16[3];
+    const unsigned blocks = unsigned(std::min<size_t>((words + 255) / 256, 148 * 8));
+    SPCONV_CUDA_TRY(launch_chained(k_fill_regions, dim3(blocks), dim3(256), stream, fr));
+  }
 
   if (known_outputs) {
     // Every size is known up front (submanifold: n_out = n; inverse: the fine positions), so the whole map including
@@ -1707,8 +1738,6 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     // The number of output rows is only known on the device: one wait for the sizes, a second one at the end
     // for the tile plan's block count.
     const int pad = d * ((K - 1) / 2);
-    SPCONV_CUDA_TRY(cudaMemsetAsync(keys2, 0xFF, size_t(cap2) * 8, stream));
-    SPCONV_CUDA_TRY(cudaMemsetAsync(owner_cid, 0x7F, size_t(cap2) * 4, stream));
     SPCONV_CUDA_TRY(launch_chained(k_insert, dim3(nblk), dim3(kBlock), stream, coords4, int(n), table1, cap1 - 1, d_status,
                                    static_cast<int4*>(nullptr), static_cast<uint32_t*>(nullptr)));
     SPCONV_CUDA_TRY(launch_chained(k_strided_candidates, grid_kn, dim3(kBlock), stream, coords4, int(n), K, s, d, pad, keys2, owner_cid,
