@@ -1638,10 +1638,12 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   if (known_outputs) {
     // Every size is known up front (submanifold: n_out = n; inverse: the fine positions), so the whole map including
     // the tile plan is enqueued before the host waits once, for the error word and the pair count.
-    { const int e = allocate_map_arrays(nq); if (e != SPCONV_OK) return e; }
+    // (the insert is enqueued before the handle's arrays are allocated where it does not write into them: the device
+    // starts a build when its first kernels arrive, and every host call in front of them is time it stands idle)
+    if (!rows_table) { const int e = allocate_map_arrays(nq); if (e != SPCONV_OK) return e; }
     SPCONV_STAGE(stages, "alloc+memset");
     SPCONV_HOST_TL("allocs+memsets");
-    int4* out_coords4 = reinterpret_cast<int4*>(km->d.out_coords);
+    int4* out_coords4 = reinterpret_cast<int4*>(km->d.out_coords);   // (null until the arrays exist)
     if (n > 0 && dense_grid != nullptr)
       SPCONV_CUDA_TRY(launch_chained(k_insert_dense, dim3(nblk_in), dim3(kBlock), stream, coords4, int(n), reinterpret_cast<int32_t*>(table1),
                                      grid_dims, d_status));
@@ -1650,6 +1652,8 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
                                      (submanifold && !rows_table) ? out_coords4 : static_cast<int4*>(nullptr), occ));
     SPCONV_STAGE(stages, "insert");
     if (rows_table) {
+      { const int e = allocate_map_arrays(nq); if (e != SPCONV_OK) return e; }
+      out_coords4 = reinterpret_cast<int4*>(km->d.out_coords);
       // every offset of a row in one thread; also copies the rows' coordinates into the handle
       auto probe_rows = [&](auto kernel) {
         return launch_chained(kernel, dim3(nblk), dim3(kBlock), stream, qcoords4, int(nq), d, s, static_cast<const LocSlot*>(table1),
