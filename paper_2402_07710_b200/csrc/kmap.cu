@@ -851,6 +851,43 @@ __global__ void k_report_totals(const int64_t* __restrict__ totals, int totals_w
 __device__ void schedule_tiles_block(const uint32_t* __restrict__ tile_mask, int n_tiles, int mask_words, int kvol,
                                      int32_t* __restrict__ sorted_tiles, uint32_t* __restrict__ status_words);
 
+// The same schedule (tiles in descending order of their block count) when every tile has already taken its place
+// among the tiles of its count (tile_within, from an atomic counter per count: class_cnt, at most 31 blocks per tile):
+// the last block only turns the 32 counts into list positions and writes each record where it belongs.  Tiles of equal
+// count come in the order their blocks finished; the forward's result does not depend on the schedule.
+__device__ __forceinline__ void schedule_from_ranks(const uint32_t* __restrict__ tile_mask, const int32_t* __restrict__ tile_within,
+                                                    const unsigned* __restrict__ class_cnt, int n_tiles,
+                                                    int32_t* __restrict__ sorted_tiles, uint32_t* __restrict__ status_words) {
+  __shared__ int s_base[32];
+  const int tid = int(threadIdx.x), T = int(blockDim.x);
+  if (tid < 16) status_words[tid] = 0u;   // the forward kernels' status record starts clean
+  constexpr int kKeep = 8;
+  uint32_t m[kKeep];
+  int32_t w[kKeep];
+#pragma unroll
+  for (int i = 0; i < kKeep; ++i) {   // all reads in flight together, beside the counts'
+    const int t = tid + i * T;
+    m[i] = t < n_tiles ? __ldcg(tile_mask + t) : 0u;
+    w[i] = t < n_tiles ? __ldcg(tile_within + t) : 0;
+  }
+  if (tid < 32) {
+    const int c = int(__ldcg(class_cnt + tid));
+    int incl = c;   // sum of the counts of this class and all heavier ones
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) { const int u = __shfl_down_sync(0xffffffffu, incl, off); if (tid + off < 32) incl += u; }
+    s_base[tid] = incl - c;
+  }
+  __syncthreads();
+  auto place = [&](int t, uint32_t mask, int32_t within) {
+    int32_t* rec = sorted_tiles + size_t(s_base[__popc(mask)] + within) * 2;
+    rec[0] = t;
+    rec[1] = int32_t(mask);
+  };
+#pragma unroll
+  for (int i = 0; i < kKeep; ++i) if (tid + i * T < n_tiles) place(tid + i * T, m[i], w[i]);
+  for (int t = tid + kKeep * T; t < n_tiles; t += T) place(t, __ldcg(tile_mask + t), __ldcg(tile_within + t));
+}
+
 // SMALL (kvol <= 32): the thread's 27-odd table entries are fetched up front, so the block pays one memory
 // latency instead of one per offset.
 template <bool SMALL>
@@ -964,7 +1001,8 @@ k_tile_plan_rows(const int32_t* __restrict__ tile_rows, const int32_t* __restric
                  int32_t* __restrict__ tile_nbr, uint8_t* __restrict__ tile_crow, uint32_t* __restrict__ tile_mask,
                  uint32_t* __restrict__ tile_absent, unsigned long long* __restrict__ block_counter,
                  unsigned* __restrict__ tiles_done, int32_t* __restrict__ sorted_tiles, uint32_t* __restrict__ status_words,
-                 const int64_t* __restrict__ totals, int totals_words, int64_t* __restrict__ host_totals, int report_from_counts) {
+                 const int64_t* __restrict__ totals, int totals_words, int64_t* __restrict__ host_totals, int report_from_counts,
+                 unsigned* __restrict__ class_cnt, int32_t* __restrict__ tile_within) {
   chain_begin();
   SPCONV_TL(6);
   __shared__ __align__(16) int32_t s_nbr[32][kPlanNbrPitch];
@@ -1018,6 +1056,8 @@ k_tile_plan_rows(const int32_t* __restrict__ tile_rows, const int32_t* __restric
   if (tid == 0) {
     tile_mask[t] = word;
     atomicAdd(block_counter, (unsigned long long)__popc(word));
+    // the tile's place among the tiles with the same number of blocks: all the last block needs to order the tiles
+    if (class_cnt != nullptr) tile_within[t] = int32_t(atomicAdd(&class_cnt[__popc(word)], 1u));
   }
   // The block that finishes last orders the tiles for the forward's schedule and reports to the host (see k_tile_plan).
   __threadfence();
@@ -1026,7 +1066,8 @@ k_tile_plan_rows(const int32_t* __restrict__ tile_rows, const int32_t* __restric
   __syncthreads();
   if (last_block) {
     __threadfence();
-    schedule_tiles_block(tile_mask, int(gridDim.x), 1, kvol, sorted_tiles, status_words);
+    if (class_cnt != nullptr) schedule_from_ranks(tile_mask, tile_within, class_cnt, int(gridDim.x), sorted_tiles, status_words);
+    else schedule_tiles_block(tile_mask, int(gridDim.x), 1, kvol, sorted_tiles, status_words);
     if (host_totals != nullptr) {
       for (int i = threadIdx.x; i < totals_words; i += blockDim.x) host_totals[i] = __ldcg(totals + i);
 #ifdef SPCONV_KMAP_TIMELINE
@@ -1423,7 +1464,8 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     if (!plan_sorted) return size_t(0);
     cub::DeviceRadixSort::SortPairs(nullptr, *cub_bytes, static_cast<uint32_t*>(nullptr), static_cast<uint32_t*>(nullptr),
                                     static_cast<int32_t*>(nullptr), static_cast<int32_t*>(nullptr), int(items), sort_begin_bit, kvol, stream);
-    return pad256(*cub_bytes) + pad256(size_t(items) * 4) * 4 + pad256((size_t(items) / (kSortThreads * kSortItemsSmall) + 8) * 1024) + 1024;
+    return pad256(*cub_bytes) + pad256(size_t(items) * 4) * 4 + pad256((size_t(items) / (kSortThreads * kSortItemsSmall) + 8) * 1024) +
+           pad256((size_t(items) / kTileRows + 2) * 4) + 1024;
   };
   size_t cub_bytes = 0;
   size_t scratch_bytes = pad256(std::max(size_t(cap1) * sizeof(LocSlot), dense_grid != nullptr ? size_t(dense_grid[0]) * dense_grid[1] * dense_grid[2] * dense_grid[3] * 4 : size_t(0))) +
@@ -1453,10 +1495,11 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   int64_t* excl_b = sa.take<int64_t>(M);
   // One zero-initialised block read back in one copy: totals [8] | offset_start [kvol + 1] | per-offset counts [32 x u32]
   const size_t totals_words = 8 + size_t(kvol) + 1;
-  int64_t* d_totals = sa.take<int64_t>(totals_words + 16);
+  int64_t* d_totals = sa.take<int64_t>(totals_words + 32);   // ... | per-offset counts [32 x u32] | tiles per block count [32 x u32]
   int64_t* d_offset_start = d_totals + 8;
   // (32 counters: only maps with kvol <= 32 get per-offset totals, which is also where the tile plan sorts by them)
   unsigned* d_offset_cnt = kvol <= 32 ? reinterpret_cast<unsigned*>(d_totals + totals_words) : nullptr;
+  unsigned* d_class_cnt = kvol <= 31 ? reinterpret_cast<unsigned*>(d_totals + totals_words + 16) : nullptr;
   int8_t* d_bitpos = sa.take<int8_t>(32);
   uint32_t* d_status = reinterpret_cast<uint32_t*>(d_totals + 2);
   unsigned long long* d_tile_blocks = reinterpret_cast<unsigned long long*>(d_totals + 3);
@@ -1559,11 +1602,14 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     }
     SPCONV_STAGE(stages, "sort");
     if (after_sort) { const int e = after_sort(); if (e != SPCONV_OK) return e; }
-    if (plan_rows != nullptr)
+    if (plan_rows != nullptr) {
+      int32_t* tile_within = (plan_sorted && d_class_cnt != nullptr) ? ta.take<int32_t>(size_t(km->n_tiles)) : nullptr;
       SPCONV_CUDA_TRY(launch_chained(k_tile_plan_rows, dim3(km->n_tiles), dim3(kTileRows), stream, static_cast<const int32_t*>(km->d.tile_rows),
                                      plan_rows, kvol, km->d.tile_nbr, km->d.tile_crow, km->d.tile_mask, km->d.tile_absent, d_tile_blocks,
                                      d_tiles_done, km->d.sorted_tiles, km->d.status, static_cast<const int64_t*>(d_totals),
-                                     int(totals_words), flag_target, counts_based ? 1 : 0));
+                                     int(totals_words), flag_target, counts_based ? 1 : 0,
+                                     tile_within != nullptr ? d_class_cnt : static_cast<unsigned*>(nullptr), tile_within));
+    }
     else if (kvol <= 32)
       SPCONV_CUDA_TRY(launch_chained(k_tile_plan<true>, dim3(km->n_tiles), dim3(kTileRows), stream, km->d.tile_rows, km->d.nbr, no, kvol,
                                      km->mask_words, km->d.tile_nbr, km->d.tile_crow, km->d.tile_mask, km->d.tile_absent, d_tile_blocks,
@@ -1624,7 +1670,7 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
   {  // (every region starts on a 256-byte boundary of the arena and is followed by padding up to the next one, so
      // rounding a size up to 16 bytes stays inside its own padding)
     FillRegions fr = {};
-    fr.ptr[0] = reinterpret_cast<uint4*>(d_totals); fr.count16[0] = ((totals_words + 16) * sizeof(int64_t) + 15) / 16; fr.value[0] = 0u;
+    fr.ptr[0] = reinterpret_cast<uint4*>(d_totals); fr.count16[0] = ((totals_words + 32) * sizeof(int64_t) + 15) / 16; fr.value[0] = 0u;
     fr.ptr[1] = reinterpret_cast<uint4*>(table1); fr.count16[1] = (table_fill_bytes + 15) / 16; fr.value[1] = 0xFFFFFFFFu;
     if (!known_outputs) {
       fr.ptr[2] = reinterpret_cast<uint4*>(keys2); fr.count16[2] = size_t(cap2) * 8 / 16; fr.value[2] = 0xFFFFFFFFu;
