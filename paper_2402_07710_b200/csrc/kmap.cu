@@ -1812,11 +1812,7 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     { const int e = wait_for_report(); if (e != SPCONV_OK) return e; }
     { const int e = allocate_map_arrays(h_totals[0]); if (e != SPCONV_OK) return e; }
     const int64_t no = km->n_out;
-    SPCONV_CUDA_TRY(cudaMemsetAsync(km->d.nbr, 0xFF, size_t(kvol) * no * 4, stream));
     { const int e = allocate_pairs(km->total_pairs); if (e != SPCONV_OK) return e; }
-    SPCONV_CUDA_TRY(launch_chained(k_owner_assign, grid_kn, dim3(kBlock), stream, static_cast<const int32_t*>(cand_slot),
-                                   static_cast<const int32_t*>(owner_cid), static_cast<const uint64_t*>(keys2), int(n),
-                                   static_cast<const int64_t*>(excl_b), slot_out, reinterpret_cast<int4*>(km->d.out_coords)));
     Scratch sort_scratch;
     sort_scratch.stream = stream;
     size_t cub2 = 0;
@@ -1825,9 +1821,18 @@ int build_kmap_impl(const int32_t* coords, int64_t n, int stride, int dilation, 
     Arena ta{static_cast<char*>(sort_scratch.ptr), bytes, 0};
     if (rows_table) {
       nbr_rows = ta.take<int32_t>(size_t(no) * 32);
-      SPCONV_CUDA_TRY(cudaMemsetAsync(nbr_rows, 0xFF, size_t(no) * 128, stream));
       plan_rows = nbr_rows;
     }
+    {  // both layouts of the offset table start as "no input row" (-1); one kernel in the chain, as at the start of a build
+      FillRegions fr = {};
+      fr.ptr[0] = reinterpret_cast<uint4*>(km->d.nbr); fr.count16[0] = (size_t(kvol) * no * 4 + 15) / 16; fr.value[0] = 0xFFFFFFFFu;
+      if (nbr_rows != nullptr) { fr.ptr[1] = reinterpret_cast<uint4*>(nbr_rows); fr.count16[1] = size_t(no) * 128 / 16; fr.value[1] = 0xFFFFFFFFu; }
+      const size_t words = fr.count16[0] + fr.count16[1];
+      SPCONV_CUDA_TRY(launch_chained(k_fill_regions, dim3(unsigned(std::min<size_t>((words + 255) / 256, 148 * 8))), dim3(256), stream, fr));
+    }
+    SPCONV_CUDA_TRY(launch_chained(k_owner_assign, grid_kn, dim3(kBlock), stream, static_cast<const int32_t*>(cand_slot),
+                                   static_cast<const int32_t*>(owner_cid), static_cast<const uint64_t*>(keys2), int(n),
+                                   static_cast<const int64_t*>(excl_b), slot_out, reinterpret_cast<int4*>(km->d.out_coords)));
     SPCONV_CUDA_TRY(launch_chained(k_strided_emit, grid_kn, dim3(kBlock), stream, static_cast<const int32_t*>(cand_slot),
                                    static_cast<const int32_t*>(slot_out), int(n), km->n_out, static_cast<const int64_t*>(excl_a),
                                    km->d.nbr, km->d.pair_in, km->d.pair_out, nbr_rows));
