@@ -457,8 +457,16 @@ __device__ void scan_counts_block(const int32_t* __restrict__ cnt, int64_t M, in
   const int tid = threadIdx.x;
   const int64_t chunk = (M + THREADS - 1) / THREADS;
   const int64_t beg = min(int64_t(tid) * chunk, M), end = min(beg + chunk, M);
+  // The first kKeep counts of a thread's chunk are read together and kept (a LiDAR-sized map has 9 per thread: one round
+  // trip to memory instead of one per count, in each of the two passes).
+  constexpr int kKeep = 16;
+  int32_t keep[kKeep];
+#pragma unroll
+  for (int i = 0; i < kKeep; ++i) keep[i] = beg + i < end ? cnt[beg + i] : 0;
   int64_t sum = 0;
-  for (int64_t i = beg; i < end; ++i) sum += cnt[i];
+#pragma unroll
+  for (int i = 0; i < kKeep; ++i) sum += keep[i];
+  for (int64_t i = beg + kKeep; i < end; ++i) sum += cnt[i];
   s[tid] = sum;
   __syncthreads();
   for (int off = 1; off < THREADS; off <<= 1) {
@@ -468,7 +476,9 @@ __device__ void scan_counts_block(const int32_t* __restrict__ cnt, int64_t M, in
     __syncthreads();
   }
   int64_t run = s[tid] - sum;
-  for (int64_t i = beg; i < end; ++i) { excl[i] = run; run += cnt[i]; }
+#pragma unroll
+  for (int i = 0; i < kKeep; ++i) if (beg + i < end) { excl[beg + i] = run; run += keep[i]; }
+  for (int64_t i = beg + kKeep; i < end; ++i) { excl[i] = run; run += cnt[i]; }
   __syncthreads();
   if (offset_start != nullptr) {
     for (int k = tid; k < kvol; k += THREADS) offset_start[k] = excl[int64_t(k) * nblk];
@@ -481,7 +491,7 @@ __device__ void scan_counts_block(const int32_t* __restrict__ cnt, int64_t M, in
   }
 }
 
-__global__ void k_scan_counts(const int32_t* __restrict__ cnt, int64_t M, int64_t* __restrict__ excl, int nblk,
+__global__ void __launch_bounds__(1024) k_scan_counts(const int32_t* __restrict__ cnt, int64_t M, int64_t* __restrict__ excl, int nblk,
                               int kvol, int64_t* __restrict__ offset_start, int64_t* __restrict__ total_out,
                               int8_t* __restrict__ bitpos) {
   chain_begin();
