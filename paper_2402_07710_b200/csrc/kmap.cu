@@ -1114,9 +1114,9 @@ k_tile_plan_rows(const int32_t* __restrict__ tile_rows, const int32_t* __restric
 
 // Schedule of the tensor-core forward: tiles in descending order of their block count, tiles of equal count in
 // ascending tile order (a stable counting sort by one thread block), so that dealing them out serpentine over the
-// CTAs gives every CTA nearly the same number of blocks and the same tiles on every run (the forward may
-// accumulate a CTA's heaviest tile in two parts, so which tiles share a CTA shows in the last bits of the result).
-// Thread i owns the contiguous chunk of tiles [i * chunk, (i + 1) * chunk).  Kernel volumes beyond 31 offsets
+// CTAs gives every CTA nearly the same number of blocks.  Used where the tiles have not taken their places within
+// their count class while the plan's blocks ran (see schedule_from_ranks); the forward's result does not depend on the
+// schedule.  Thread i owns the contiguous chunk of tiles [i * chunk, (i + 1) * chunk).  Kernel volumes beyond 31 offsets
 // (more count classes than the per-thread counters hold) fall back to an unordered placement within a class.
 __device__ void schedule_tiles_block(const uint32_t* __restrict__ tile_mask, int n_tiles, int mask_words, int kvol,
                                      int32_t* __restrict__ sorted_tiles, uint32_t* __restrict__ status_words) {
